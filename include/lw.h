@@ -109,7 +109,22 @@ int lw_dequant(int fmt, const void* W_blocks, int64_t n, float* out, void* strea
  *           aligned, read-only.
  * X: device, batch * cols floats, each activation vector contiguous, 16-byte aligned, read-only.
  * Y: device, batch * rows floats, 16-byte aligned, fully overwritten (never accumulated into).
- * Asynchronous on `stream`; results satisfy |y - y_exact| <= 1e-4 * sum|w*x| + 1e-6. */
+ * Asynchronous on `stream`.
+ * Accuracy.  With w the decoded weights and S = sum_k |w_k x_k|, every result satisfies
+ *     |y - y_exact| <= 1e-4 * S + 1e-6 + E .
+ * E = 0 for LW_VARIANT_GENERIC and for f16 (each weight is decoded exactly and then multiplied: plain fp32
+ * accumulation), for any finite input.  The streaming variants multiply the integer codes first and apply
+ * block scales and offsets to the sums, and LW_VARIANT_IDOT holds the activations as block fixed point
+ * (23 bits + sign relative to the largest magnitude in each run of 16 or 32), so an activation that is
+ * huge compared with its neighbours and meets a weight that is zero or nearly so leaves an absolute error
+ * that S does not cover.  For them
+ *     E = c * sum_k What_k * A_k ,   c = 2^-18 (IDOT, the default for the quantised formats), 2^-16 (STREAM),
+ * where, over the aligned run of 32 columns that contains k, A_k is the largest |x| and What_k the largest
+ * decoded |w|.  This holds for weights made by lw_quantize, and for any block whose scale * code and offset
+ * terms are at most four times its largest decoded magnitude.  The constants are worst-case figures (the
+ * largest c observed on inputs built to provoke the term is 2^-26 for IDOT and 2^-22 for STREAM); on
+ * Gaussian activations and weights the measured error stays below 0.001 of 1e-4 * S.
+ * A NaN or Inf activation makes every output of its column's rows non-finite in every variant. */
 int lw_matvec(int fmt, const void* W_blocks, int64_t rows, int64_t cols,
               const float* X, float* Y, int batch, void* stream);
 
@@ -143,13 +158,16 @@ typedef enum {
     LW_VARIANT_AUTO = 0,
     LW_VARIANT_GENERIC = 1, /* one warp per row, plain loads; any legal shape and batch */
     LW_VARIANT_STREAM = 2,  /* bulk-copy ring into shared memory, fp32 activations held in registers, one
-                               512-thread CTA per SM; needs cols % 256 == 0 and cols <= 16384; batch 1 */
+                               512-thread CTA per SM; needs cols % 256 == 0, cols <= 16384 and rows that are
+                               whole 16-byte pieces; batch 1.  Exists for f16, q8_0, q4_0 and q4_K; forced on
+                               one of the six later formats it falls back to LW_VARIANT_GENERIC */
     LW_VARIANT_IDOT = 3     /* same streaming skeleton, but activations are converted once per call to
                                24-bit block fixed point (one fp32 scale per 16 or 32 values) and the
                                products run as exact integer dot products (dp4a); error per
-                               activation <= 2^-23 of its group's largest magnitude.  q8_0, q4_0,
-                               q4_K only (f16 falls back to LW_VARIANT_STREAM).  Also has a batched
-                               form (2..16 columns, fixed-point activations kept in shared memory) */
+                               activation <= 2^-22 of its group's largest magnitude (see the accuracy
+                               statement of lw_matvec).  All nine quantised formats (f16 falls back to
+                               LW_VARIANT_STREAM).  q8_0, q4_0 and q4_K also have a batched form (2..16
+                               columns, fixed-point activations kept in shared memory) */
 } lw_variant;
 /* Process-wide; returns LW_ERR_FORMAT for an unknown value.  Also settable once at load time
  * through the environment variable LW_FORCE_VARIANT (a number).  A forced variant that does not
@@ -175,10 +193,10 @@ int lw_set_tuning(int worker_groups, int stages, int stage_kb);
  * query. */
 int lw_plan_info(int fmt, int64_t rows, int64_t cols, int* out6);
 
-/* Overlap of consecutive calls on one stream (programmatic dependent launch): when enabled, a
- * mat-vec kernel may begin streaming its weights while the previous kernel on the stream is still
- * finishing, and waits for that kernel only before it reads X or writes Y.  Enable only when
- * W_blocks is constant model data that no kernel still running on the stream writes.
+/* Overlap of consecutive calls on one stream (programmatic dependent launch): when enabled, the
+ * launches carry the programmatic-serialisation attribute, so a mat-vec kernel's CTAs may be placed and
+ * run their set-up (barrier initialisation, launch latency) while the previous kernel on the stream is
+ * still finishing; they wait for that kernel to complete before they request any of W or X or write Y.
  * Default off.  Process-wide. */
 int lw_set_overlap(int enabled);
 
@@ -241,6 +259,13 @@ int lw_attn_decode_static(int kv_fmt, const void* K_blocks, const void* V_blocks
  * never trap or spin forever: a bounded wait that gives up records a code here and the kernel
  * finishes.  This call synchronises the device.  Returns LW_OK, LW_ERR_NULL or LW_ERR_CUDA. */
 int lw_device_status(int* status_out);
+
+/* Testing aid for that fault path (the paper has no counterpart).  After lw_debug_drop_copy(u), u >= 0, the
+ * next batch-1 lw_matvec that takes a streaming kernel never requests the copy of the u-th row unit of each
+ * CTA: nothing is in flight for it, the wait for it runs out after its limit (about 0.1 s), the kernel
+ * records a fault, requests nothing further and returns; the rows of that unit and of the units after it are
+ * left unwritten.  The request is consumed by that one launch; u < 0 cancels it.  Always returns LW_OK. */
+int lw_debug_drop_copy(int unit);
 
 #ifdef __cplusplus
 }

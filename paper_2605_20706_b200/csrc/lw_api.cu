@@ -58,7 +58,10 @@ static int pick_variant(int fmt, int64_t rows, int64_t cols, int batch) {
         if (forced == LW_VARIANT_STREAM) return LW_VARIANT_GENERIC;
         return (batch <= 4 || forced == LW_VARIANT_IDOT) ? LW_VARIANT_IDOT : LW_VARIANT_GENERIC;
     }
-    if (forced == LW_VARIANT_STREAM || fmt == LW_F16) return LW_VARIANT_STREAM;
+    if (fmt == LW_F16) return LW_VARIANT_STREAM;
+    // the fp32-activation streaming family exists for q8_0, q4_0 and q4_K; for the later formats a forced
+    // STREAM falls back to the next simpler variant
+    if (forced == LW_VARIANT_STREAM) return fmt <= LW_Q4_K ? LW_VARIANT_STREAM : LW_VARIANT_GENERIC;
     return LW_VARIANT_IDOT;
 }
 
@@ -179,7 +182,9 @@ int lw_matvec_group(int fmt, int64_t cols, int n_items, const lw_group_item* ite
         if (rc != LW_OK) return rc;
     }
     const int forced = forced_variant();
-    if (forced != LW_VARIANT_GENERIC && matvec_group_supported(fmt, cols, n_items)) {
+    const bool has_fp32_stream = fmt <= LW_Q4_K;
+    if (forced != LW_VARIANT_GENERIC && !(forced == LW_VARIANT_STREAM && !has_fp32_stream) &&
+        matvec_group_supported(fmt, cols, n_items)) {
         const void* W[8];
         const float* X[8];
         float* Y[8];
@@ -244,6 +249,11 @@ int lw_plan_info(int fmt, int64_t rows, int64_t cols, int* out6) {
     if (!stream_plan_info(fmt, rows, cols, &out6[0], &out6[1], &out6[2], &out6[3], &out6[4], &out6[5])) {
         for (int i = 0; i < 6; ++i) out6[i] = 0;       // shape not covered by the streaming kernels
     }
+    return LW_OK;
+}
+
+int lw_debug_drop_copy(int unit) {
+    set_drop_unit(unit);
     return LW_OK;
 }
 

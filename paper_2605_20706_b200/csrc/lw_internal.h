@@ -38,6 +38,8 @@ int launch_matvec_stream_group(int fmt, bool integer_dot, int64_t cols, int n_it
                                cudaStream_t stream);
 // Tunables of the streaming kernels (0 = automatic) and the geometry they lead to for a shape.
 void set_stream_tuning(int worker_groups, int stages, int stage_kb);
+// Testing aid: the next single-matrix streaming launch never requests the copy of pool unit `unit` (< 0: none).
+void set_drop_unit(int unit);
 bool stream_plan_info(int fmt, int64_t rows, int64_t cols, int* groups, int* stages, int* stage_rows, int* stage_bytes,
                       int* grid, int* smem_bytes);
 // Decode attention over a quantised KV cache: shape check, parts the positions are cut into, bytes of

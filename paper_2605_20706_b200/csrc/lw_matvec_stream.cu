@@ -23,6 +23,7 @@
 #include <cuda_fp16.h>
 #include <cuda_runtime.h>
 
+#include <atomic>
 #include <cstdlib>
 #include <type_traits>
 
@@ -353,13 +354,21 @@ __device__ __forceinline__ void quantize_activations(const float* __restrict__ X
             if (run0 + j * NTHREADS >= padded) break;      // warp-uniform: whole warps drop out together
             const int run = run0 + j * NTHREADS;
             const bool valid = run < runs;
-            float amax = 0.f;
+            float amax = 0.f, nonfinite = 0.f;
 #pragma unroll
-            for (int i = 0; i < 16; ++i) amax = fmaxf(amax, fabsf(v[j][i]));
-            if (GROUP == 32) amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, 1));
+            for (int i = 0; i < 16; ++i) {
+                amax = fmaxf(amax, fabsf(v[j][i]));
+                nonfinite = fmaf(v[j][i], 0.f, nonfinite);      // stays 0 unless a value is NaN or Inf
+            }
+            if (GROUP == 32) {
+                amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, 1));
+                nonfinite += __shfl_xor_sync(0xFFFFFFFFu, nonfinite, 1);
+            }
+            // A NaN or Inf activation must reach every output it touches (as in fp32 arithmetic): the
+            // maximum above drops NaNs, so the group's scale is made NaN explicitly.
             const bool nonzero = amax > 1e-30f;
-            const float d = nonzero ? amax / 4194303.f : 0.f;
-            const float inv = nonzero ? 4194303.f / amax : 0.f;
+            const float d = nonfinite != 0.f ? nonfinite : (nonzero ? amax / 4194303.f : 0.f);
+            const float inv = nonzero && amax <= 3.0e38f ? 4194303.f / amax : 0.f;
             int q[16];
             int total = 0;
 #pragma unroll
@@ -1158,6 +1167,7 @@ struct StreamParams {
         int rows_per_cta;
     } items[kMaxGroup];
     uint32_t xq_col_words;   // words between the fixed-point activations of consecutive columns
+    int drop_unit;           // testing aid: the unit (index in the CTA's pool) whose copy is never requested; -1 = none
 };
 
 // Shared-memory float index of activation k after padding (4 floats after every kXChunk).
@@ -1235,6 +1245,7 @@ __global__ void __launch_bounds__(NG* kThreads, NG == 1 ? T::kMinCtas : 1)
     uint64_t* xbar = reinterpret_cast<uint64_t*>(smem + 64);
     volatile int* timed_out = reinterpret_cast<volatile int*>(smem + 72);
     int* unit_counter = reinterpret_cast<int*>(smem + 76);
+    volatile int* copy_dropped = reinterpret_cast<volatile int*>(smem + 336);    // behind the unit records
     const int partial_stride = p.stage_rows * p.units_per_row;      // floats per buffer
     float* xs = reinterpret_cast<float*>(smem + p.x_off);
 
@@ -1284,6 +1295,7 @@ __global__ void __launch_bounds__(NG* kThreads, NG == 1 ? T::kMinCtas : 1)
         mbar_init(xbar, 1);
         *timed_out = 0;
         *unit_counter = 0;
+        *copy_dropped = 0;
         fence_barrier_init();
     }
     __syncthreads();
@@ -1299,19 +1311,24 @@ __global__ void __launch_bounds__(NG* kThreads, NG == 1 ? T::kMinCtas : 1)
         if constexpr (NG == 1) k = next_unit++;
         else k = atomicAdd(unit_counter, 1);
         int begin = 0, n = 0;
-        if (k < n_units) {
+        if (k < n_units && *copy_dropped == 0) {
             begin = k < n_short ? k * rows_per_wave : short_rows + (k - n_short) * stage_rows;
             n = rows_here - begin;
             const int cap = k < n_short ? rows_per_wave : stage_rows;
             if (n > cap) n = cap;
         }
+        // Testing aid: the copy of one unit is never requested, so the wait for it must run out.  Nothing
+        // is queued in the CTA after that (no later copy can land in a slot whose barrier is out of
+        // step), and the rows of the units left over are not computed.
+        const bool drop = n > 0 && k == p.drop_unit;
+        if (drop) *copy_dropped = 1;
         {
             uint8_t* rec = smem + rec_base + 16u * (uint32_t)(claims & (kUnitRecords - 1));
             *reinterpret_cast<float**>(rec) = Ym + row0 + begin;
             *reinterpret_cast<int*>(rec + 8) = n;
             ++claims;
         }
-        if (n > 0) {
+        if (n > 0 && !drop) {
             const uint32_t bytes = (uint32_t)(n * row_bytes);
             mbar_expect_tx(&full[slot], bytes);
             bulk_load(ring + slot * stage_stride, wbase + (int64_t)begin * row_bytes, bytes, &full[slot], policy);
@@ -1686,6 +1703,13 @@ Tuning& tuning_storage() {
 }
 const Tuning& tuning() { return tuning_storage(); }
 
+// Testing aid (lw_debug_drop_copy): the next batch-1 streaming launch leaves out the copy of one unit.
+std::atomic<int>& drop_unit_storage() {
+    static std::atomic<int> v{-1};
+    return v;
+}
+int take_drop_unit() { return drop_unit_storage().exchange(-1); }
+
 constexpr size_t kSmemPerSm = 233472;      // 228 KB of shared memory per SM, 1 KB reserved per CTA
 constexpr size_t kSmemMaxCta = 227 * 1024;    // largest opt-in dynamic shared memory of a CTA
 
@@ -1769,6 +1793,7 @@ Plan make_plan(int fmt, bool integer_dot, int64_t rows, int64_t cols, int num_sm
     pl.p.stage_stride = best_stride;
     pl.p.x_off = (uint32_t)best_x_off;
     pl.p.ring_off = (uint32_t)best_ring_off;
+    pl.p.drop_unit = -1;
     pl.groups = groups;
     pl.grid = (unsigned)grid;
     pl.smem_bytes = best_smem;
@@ -1888,6 +1913,8 @@ int batched_columns(int fmt, int64_t rows, int64_t cols) {
 }
 
 }  // namespace
+
+void set_drop_unit(int unit) { drop_unit_storage().store(unit < 0 ? -1 : unit); }
 
 void set_stream_tuning(int worker_groups, int stages, int stage_kb) {
     Tuning& t = tuning_storage();
@@ -2017,6 +2044,7 @@ int launch_matvec_stream(int fmt, bool integer_dot, const void* W, int64_t rows,
     pl.p.X = X;
     pl.p.Y = Y;
     pl.p.fault = fault;
+    pl.p.drop_unit = take_drop_unit();
     switch (fmt) {
         case LW_F16:
             return launch_one<StreamF16>(pl, overlap, stream);

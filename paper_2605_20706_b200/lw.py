@@ -30,7 +30,8 @@ LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "liblw.so")
 EXPORTS = ("lw_block_elems", "lw_block_bytes", "lw_row_bytes", "lw_status_string", "lw_quantize",
            "lw_dequant", "lw_matvec", "lw_matvec_group", "lw_matvec_host", "lw_set_variant", "lw_query_variant",
            "lw_set_overlap", "lw_device_status", "lw_set_tuning", "lw_plan_info", "lw_attn_decode",
-           "lw_attn_workspace_bytes", "lw_attn_decode_static", "lw_set_attn_variant", "lw_query_attn_variant")
+           "lw_attn_workspace_bytes", "lw_attn_decode_static", "lw_set_attn_variant", "lw_query_attn_variant",
+           "lw_debug_drop_copy")
 
 _lib = None
 
@@ -73,6 +74,7 @@ def lib() -> ctypes.CDLL:
     L.lw_attn_decode.argtypes = [c_int, vp, vp, vp, vp, i64, i64, i64, i64, ctypes.c_float, vp, i64, vp]
     L.lw_set_attn_variant.restype, L.lw_set_attn_variant.argtypes = c_int, [c_int]
     L.lw_query_attn_variant.restype, L.lw_query_attn_variant.argtypes = c_int, [c_int, i64, i64, i64, i64]
+    L.lw_debug_drop_copy.restype, L.lw_debug_drop_copy.argtypes = c_int, [c_int]
     L.lw_attn_decode_static.restype = c_int
     L.lw_attn_decode_static.argtypes = [c_int, vp, vp, vp, vp, i64, i64, i64, i64, ctypes.c_float, vp]
     _lib = L
@@ -223,6 +225,11 @@ def plan_info(fmt: int, rows: int, cols: int) -> dict:
     _check(lib().lw_plan_info(fmt, rows, cols, ctypes.cast(out, ctypes.c_void_p)), "lw_plan_info")
     keys = ("worker_groups", "stages", "stage_rows", "stage_bytes", "ctas", "smem_bytes")
     return dict(zip(keys, list(out)))
+
+
+def debug_drop_copy(unit: int) -> None:
+    """Testing aid: the next single-matrix streaming mat-vec never requests the copy of pool unit `unit`."""
+    _check(lib().lw_debug_drop_copy(unit), "lw_debug_drop_copy")
 
 
 def device_status() -> int:

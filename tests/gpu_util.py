@@ -1,4 +1,6 @@
-"""Helpers shared by the GPU parity tests: seeded inputs, oracle-quantised weights, tolerance."""
+"""Helpers shared by the GPU parity tests: seeded inputs, oracle-quantised weights, tolerance, and
+output buffers with guard words on both sides (the bounds check of these tests: a kernel that writes
+one element before or past its output changes a guard word)."""
 from concurrent.futures import ThreadPoolExecutor
 import os
 
@@ -45,3 +47,32 @@ def check_matvec(y_gpu, y_ref, s_ref, what=""):
         nmse = float(((y_gpu - y_ref) ** 2).sum() / denom)
         assert nmse <= NMSE_MAX, "%s: NMSE %.3g" % (what, nmse)
     return worst
+
+
+GUARD_WORDS = 64                  # 256 bytes on each side: keeps the 16-byte alignment the library asks for
+GUARD_PATTERN = 0x5AC3A55A        # as int32; as a float it is a finite number no kernel here produces
+
+
+class Guarded:
+    """A device buffer of `n` 4-byte elements between two runs of guard words.  `.t` is the tensor to hand to
+    the library (viewed as `dtype`, shaped `shape`); `.check()` asserts that no guard word changed."""
+
+    def __init__(self, shape, fill=float("nan"), dtype=None):
+        import torch
+        dtype = dtype or torch.float32
+        assert dtype in (torch.float32, torch.int32)
+        shape = (shape,) if isinstance(shape, int) else tuple(shape)
+        n = int(np.prod(shape))
+        self.n = n
+        self.raw = torch.full((n + 2 * GUARD_WORDS,), GUARD_PATTERN, dtype=torch.int32, device="cuda")
+        self.t = self.raw[GUARD_WORDS:GUARD_WORDS + n].view(dtype).view(shape)
+        if fill is not None:
+            self.t.fill_(fill)
+
+    def check(self, what=""):
+        import torch
+        torch.cuda.synchronize()
+        lo = self.raw[:GUARD_WORDS].cpu().numpy()
+        hi = self.raw[GUARD_WORDS + self.n:].cpu().numpy()
+        assert (lo == GUARD_PATTERN).all(), "%s: write before the start of the buffer" % what
+        assert (hi == GUARD_PATTERN).all(), "%s: write past the end of the buffer" % what

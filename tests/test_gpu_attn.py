@@ -6,6 +6,8 @@ import pytest
 import oracle
 from paper_2605_20706_b200 import lw, synth
 
+from gpu_util import Guarded
+
 torch = pytest.importorskip("torch")
 pytestmark = pytest.mark.gpu
 
@@ -32,14 +34,15 @@ def gpu_attn(fmt, K, V, q, n_head, n_kv, hd, n_pos, scale, repeat=1, variant=lw.
     k = torch.from_numpy(K).cuda()
     v = torch.from_numpy(V).cuda()
     qd = torch.from_numpy(np.ascontiguousarray(q, dtype=np.float32)).cuda()
-    out = torch.full((n_head, hd), float("nan"), dtype=torch.float32, device="cuda")
-    ws = torch.full((lw.attn_workspace_bytes(n_head, n_kv, hd, n_pos) // 4,), float("nan"), dtype=torch.float32,
-                    device="cuda")
+    out = Guarded((n_head, hd))                # NaN-filled, guard words on both sides
+    ws = Guarded(lw.attn_workspace_bytes(n_head, n_kv, hd, n_pos) // 4)
     for _ in range(repeat):
-        lw.attn_decode(fmt, k, v, qd, out, n_head, n_kv, hd, n_pos, scale, ws)
+        lw.attn_decode(fmt, k, v, qd, out.t, n_head, n_kv, hd, n_pos, scale, ws.t)
     torch.cuda.synchronize()
     assert lw.device_status() == 0
-    return out.cpu().numpy()
+    out.check("attention output")
+    ws.check("attention workspace")
+    return out.t.cpu().numpy()
 
 
 def check(out, ref, S, what):

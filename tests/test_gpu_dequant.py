@@ -5,6 +5,8 @@ import pytest
 import oracle
 from paper_2605_20706_b200 import lw, synth
 
+from gpu_util import Guarded
+
 torch = pytest.importorskip("torch")
 pytestmark = pytest.mark.gpu
 
@@ -13,10 +15,11 @@ FMTS = [lw.F16, lw.Q8_0, lw.Q4_0, lw.Q4_K, lw.Q6_K, lw.Q5_K, lw.Q2_K, lw.Q4_1, l
 
 def _gpu_dequant(fmt, blocks, n):
     w = torch.from_numpy(blocks).cuda()
-    out = torch.full((n,), float("nan"), dtype=torch.float32, device="cuda")
-    lw.dequant(fmt, w, n, out)
+    out = Guarded(n)                           # NaN-filled, guard words on both sides
+    lw.dequant(fmt, w, n, out.t)
     torch.cuda.synchronize()
-    return out.cpu().numpy()
+    out.check("dequant output")
+    return out.t.cpu().numpy()
 
 
 @pytest.mark.parametrize("fmt", FMTS)

@@ -8,7 +8,7 @@ import pytest
 import oracle
 from paper_2605_20706_b200 import lw, synth
 
-from gpu_util import check_matvec, quantized_weights
+from gpu_util import Guarded, check_matvec, quantized_weights
 
 torch = pytest.importorskip("torch")
 pytestmark = pytest.mark.gpu
@@ -32,7 +32,8 @@ def _run_case(fmt, rows, cols, seed, outlier_p):
     X = synth.activations(seed, rows % 89, 1, cols)
     w = torch.from_numpy(blocks).cuda()
     x = torch.from_numpy(X).cuda()
-    y = torch.full((1, rows), float("nan"), dtype=torch.float32, device="cuda")
+    guarded = Guarded((1, rows))
+    y = guarded.t
     lw.set_variant(lw.VARIANT_AUTO)
     lw.set_overlap(True)
     try:
@@ -50,6 +51,7 @@ def _run_case(fmt, rows, cols, seed, outlier_p):
     finally:
         lw.set_overlap(False)
     assert lw.device_status() == 0
+    guarded.check("Y of fmt %d %dx%d" % (fmt, rows, cols))
     got = y.cpu().numpy()
     assert np.isfinite(got).all()
     idx = _sample_rows(rows, np.random.default_rng(seed))
@@ -77,9 +79,11 @@ def test_llama8b_gate_batched(batch):
     X = synth.activations(5, 7, batch, cols)
     w = torch.from_numpy(blocks).cuda()
     x = torch.from_numpy(X).cuda()
-    y = torch.full((batch, rows), float("nan"), dtype=torch.float32, device="cuda")
+    guarded = Guarded((batch, rows))
+    y = guarded.t
     lw.matvec(fmt, w, rows, cols, x, y, batch)
     torch.cuda.synchronize()
+    guarded.check("Y of the batched gate")
     idx = _sample_rows(rows, np.random.default_rng(batch), n=400)
     y_ref, s_ref = oracle.matvec(fmt, blocks, rows, cols, X, batch, nthreads=8, row_idx=idx)
     check_matvec(y.cpu().numpy()[:, idx], y_ref, s_ref, "batched gate, batch %d" % batch)

@@ -146,6 +146,8 @@ def test_variant_controls():
     assert lw.query_variant(lw.Q8_0, 64, 32768, 1) == lw.VARIANT_GENERIC     # too wide for one CTA
     lw.set_variant(lw.VARIANT_STREAM)
     assert lw.query_variant(lw.Q4_0, 4096, 4096, 1) == lw.VARIANT_STREAM
+    for f in (lw.Q6_K, lw.Q5_K, lw.Q2_K, lw.Q4_1, lw.Q5_0, lw.Q5_1):      # no fp32-activation streaming form
+        assert lw.query_variant(f, 4096, 4096, 1) == lw.VARIANT_GENERIC
     lw.set_variant(lw.VARIANT_AUTO)
     assert lw.query_variant(lw.Q4_0, 16, 96, 1) == lw.VARIANT_GENERIC      # cols % 256 != 0
     with pytest.raises(lw.LwError):
