@@ -200,6 +200,12 @@ def run_ours(args):
     xh = X_host.numpy()
     for i, (_, r, c) in enumerate(shapes):
         xh[xoffs[i]:xoffs[i] + batch * c] = synth.activations(seed, i, batch, c).reshape(-1)
+    # q/k/v of a layer read the same activations, and so do gate/up: give them identical values
+    for i in range(1, ncalls):
+        leaf, prev = shapes[i][0].split(".")[-1], shapes[i - 1][0].split(".")[-1]
+        if (leaf, prev) in (("k", "q"), ("v", "k"), ("up", "gate")) and shapes[i][2] == shapes[i - 1][2]:
+            c = shapes[i][2]
+            xh[xoffs[i]:xoffs[i] + batch * c] = xh[xoffs[i - 1]:xoffs[i - 1] + batch * c]
     X = X_host.cuda()
     Y = torch.zeros(yt, dtype=torch.float32, device="cuda")
 
@@ -268,9 +274,25 @@ def run_ours(args):
                                 [(wptr + offs[j], shapes[j][1], xptr + 4 * xoffs[j], yptr + 4 * yoffs[j]) for j in g],
                                 stream)
 
-    grouped = batch == 1 and not args.per_call
-    enqueue_step = enqueue_grouped if grouped else enqueue_per_call
-    launches_per_step = len(groups) if grouped else ncalls
+    # Sequence issue: the whole chain in ONE lw_matvec_sequence call (persistent kernel); q/k/v and
+    # gate/up share their X; every other mat-vec is flagged dependent on what came before it.
+    seq_list = []
+    for g in groups:
+        for n, j in enumerate(g):
+            _, r, c = shapes[j]
+            x_of = g[0]          # the members of a group read the same activations
+            seq_list.append((wptr + offs[j], r, c, xptr + 4 * xoffs[x_of], yptr + 4 * yoffs[j],
+                             lw.SEQ_DEPENDENT if n == 0 else 0))
+    seq_arr = lw.seq_items(seq_list)
+    seq_ws = torch.zeros(lw.matvec_sequence_workspace_bytes() // 4, dtype=torch.int32, device="cuda")
+
+    def enqueue_sequence(stream):
+        lw.matvec_sequence(fmt_id, seq_arr, seq_ws, stream=stream)
+
+    sequence = batch == 1 and args.issue == "sequence"
+    grouped = batch == 1 and args.issue == "grouped"
+    enqueue_step = enqueue_sequence if sequence else (enqueue_grouped if grouped else enqueue_per_call)
+    launches_per_step = 1 if sequence else (len(groups) if grouped else ncalls)
 
     side = torch.cuda.Stream()
     with torch.cuda.stream(side):
@@ -778,7 +800,9 @@ def main():
     ap.add_argument("--only", default=None, help="comma-separated substrings: keep only matching mat-vecs "
                                                   "(profiling of single kernels)")
     ap.add_argument("--no-graph", action="store_true")
-    ap.add_argument("--per-call", action="store_true", help="one lw_matvec per mat-vec instead of grouped calls")
+    ap.add_argument("--issue", default="sequence", choices=["sequence", "grouped", "per-call"],
+                    help="sequence: one lw_matvec_sequence call per step; grouped: lw_matvec_group for q/k/v and "
+                         "gate/up, lw_matvec for the rest; per-call: one lw_matvec per mat-vec")
     ap.add_argument("--serial", action="store_true", help="one branch: every mat-vec waits for the previous one")
     ap.add_argument("--no-overlap", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")

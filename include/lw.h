@@ -152,6 +152,39 @@ typedef struct {
 } lw_group_item;
 int lw_matvec_group(int fmt, int64_t cols, int n_items, const lw_group_item* items, void* stream);
 
+/* A whole chain of batch-1 mat-vecs of one format in ONE launch [Sec 3.1, 3.2: the runtime groups operations
+ * into compute passes; the whole mat-vec chain of a decode step is one pass here].  The items run in the
+ * order given.  Consecutive items that read the same X (same pointer, same cols) and are not flagged
+ * dependent form one phase whose rows are shared out over all SMs together (q/k/v, gate/up).  An item
+ * flagged LW_SEQ_DEPENDENT reads (X) or overwrites (Y) memory that an earlier item of the sequence writes
+ * or reads: before it starts, every earlier item has finished device-wide (a grid-wide barrier inside the
+ * kernel).  Without the flag an item may run concurrently with its predecessors.  The kernel is persistent,
+ * one CTA per SM, launched cooperatively: the weight ring keeps filling across item boundaries (weights are
+ * constant data), so a boundary costs a barrier and the activation fetch instead of a kernel launch with a
+ * cold pipeline.
+ * Each item is what lw_matvec takes at batch 1 (W: rows * lw_row_bytes(fmt, cols) bytes; X: cols floats;
+ * Y: rows floats; all device, 16-byte aligned); n_items <= 640, at most 320 phases.
+ * workspace: device, at least lw_matvec_sequence_workspace_bytes() bytes, 16-byte aligned, owned by the
+ *           caller, need not be initialised (the call clears what it needs on `stream` first); sequences that
+ *           may run concurrently need separate workspaces.
+ * `items` is host memory, read during the call only.  Results and accuracy are those of lw_matvec.
+ * When a shape is not covered by the streaming kernels, a variant is forced, or the device cannot launch
+ * cooperatively, the items are issued one after the other with lw_matvec on `stream` (stream order then
+ * provides every dependency).  Asynchronous on `stream`; can be captured into a CUDA graph.
+ * Errors: as lw_matvec per item, LW_ERR_SHAPE for n_items outside 1..640, LW_ERR_WORKSPACE. */
+typedef struct {
+    const void* W_blocks;
+    int64_t rows;
+    int64_t cols;
+    const float* X;
+    float* Y;
+    int flags;              /* 0 or LW_SEQ_DEPENDENT */
+} lw_seq_item;
+enum { LW_SEQ_DEPENDENT = 1 };
+int64_t lw_matvec_sequence_workspace_bytes(void);
+int lw_matvec_sequence(int fmt, int n_items, const lw_seq_item* items, void* workspace, int64_t workspace_bytes,
+                       void* stream);
+
 /* Kernel-variant selection [Sec 3.2: the kernel library picks a variant from the tensor context;
  * tunable work-group and tile sizes].  LW_VARIANT_AUTO lets the launch heuristics decide. */
 typedef enum {

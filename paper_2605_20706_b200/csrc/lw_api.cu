@@ -207,6 +207,40 @@ int lw_matvec_group(int fmt, int64_t cols, int n_items, const lw_group_item* ite
     return LW_OK;
 }
 
+int64_t lw_matvec_sequence_workspace_bytes(void) { return 256; }
+
+int lw_matvec_sequence(int fmt, int n_items, const lw_seq_item* items, void* workspace, int64_t workspace_bytes,
+                       void* stream) {
+    if (lw_block_elems(fmt) == 0) return LW_ERR_FORMAT;
+    if (!items || !workspace) return LW_ERR_NULL;
+    if (n_items < 1 || n_items > 640) return LW_ERR_SHAPE;
+    if (misaligned16(workspace)) return LW_ERR_ALIGN;
+    if (workspace_bytes < lw_matvec_sequence_workspace_bytes()) return LW_ERR_WORKSPACE;
+    for (int j = 0; j < n_items; ++j) {
+        const int rc = check_matvec_args(fmt, items[j].W_blocks, items[j].rows, items[j].cols, items[j].X, items[j].Y, 1);
+        if (rc != LW_OK) return rc;
+        if (items[j].flags & ~LW_SEQ_DEPENDENT) return LW_ERR_FORMAT;
+    }
+    static int coop[64] = {0};          // 0 unknown, 1 yes, -1 no
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return LW_ERR_CUDA;
+    if (dev >= 0 && dev < 64 && coop[dev] == 0) {
+        int v = 0;
+        coop[dev] = (cudaDeviceGetAttribute(&v, cudaDevAttrCooperativeLaunch, dev) == cudaSuccess && v) ? 1 : -1;
+    }
+    const bool can = dev >= 0 && dev < 64 && coop[dev] == 1;
+    if (can && forced_variant() == LW_VARIANT_AUTO && matvec_sequence_supported(fmt, n_items, items)) {
+        const int err = launch_matvec_sequence(fmt, n_items, items, static_cast<unsigned*>(workspace),
+                                               static_cast<cudaStream_t>(stream));
+        return err == 0 ? LW_OK : LW_ERR_CUDA;
+    }
+    for (int j = 0; j < n_items; ++j) {
+        const int rc = lw_matvec(fmt, items[j].W_blocks, items[j].rows, items[j].cols, items[j].X, items[j].Y, 1, stream);
+        if (rc != LW_OK) return rc;
+    }
+    return LW_OK;
+}
+
 int lw_matvec_host(int fmt, const void* W_blocks, int64_t rows, int64_t cols, const float* X_host,
                    float* Y_host, float* X_dev, float* Y_dev, int batch, void* stream) {
     if (!X_host || !Y_host) return LW_ERR_NULL;

@@ -13,7 +13,8 @@ namespace lw {
 enum DeviceFault : int {
     FAULT_NONE = 0,
     FAULT_BULK_WAIT_TIMEOUT = 1,   // a bounded wait on a bulk-copy barrier gave up
-    FAULT_DRAIN_TIMEOUT = 2        // the end-of-kernel drain of copies in flight gave up
+    FAULT_DRAIN_TIMEOUT = 2,       // the end-of-kernel drain of copies in flight gave up
+    FAULT_GRID_BARRIER_TIMEOUT = 3 // a CTA of the sequence kernel gave up waiting for the other CTAs
 };
 
 int quantize_host(int fmt, const float* src, int64_t n, void* dst);
@@ -36,6 +37,10 @@ bool matvec_group_supported(int fmt, int64_t cols, int n_items);
 int launch_matvec_stream_group(int fmt, bool integer_dot, int64_t cols, int n_items, const void* const* W,
                                const int64_t* rows, const float* const* X, float* const* Y, bool overlap,
                                cudaStream_t stream);
+// Sequence of batch-1 mat-vecs in one persistent launch (grid-wide barrier before dependent items).
+// `counter` is a device word owned by the caller (cleared on the stream by the launch).
+bool matvec_sequence_supported(int fmt, int n_items, const lw_seq_item* items);
+int launch_matvec_sequence(int fmt, int n_items, const lw_seq_item* items, unsigned* counter, cudaStream_t stream);
 // Tunables of the streaming kernels (0 = automatic) and the geometry they lead to for a shape.
 void set_stream_tuning(int worker_groups, int stages, int stage_kb);
 // Testing aid: the next single-matrix streaming launch never requests the copy of pool unit `unit` (< 0: none).

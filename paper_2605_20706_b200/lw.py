@@ -31,7 +31,7 @@ EXPORTS = ("lw_block_elems", "lw_block_bytes", "lw_row_bytes", "lw_status_string
            "lw_dequant", "lw_matvec", "lw_matvec_group", "lw_matvec_host", "lw_set_variant", "lw_query_variant",
            "lw_set_overlap", "lw_device_status", "lw_set_tuning", "lw_plan_info", "lw_attn_decode",
            "lw_attn_workspace_bytes", "lw_attn_decode_static", "lw_set_attn_variant", "lw_query_attn_variant",
-           "lw_debug_drop_copy")
+           "lw_debug_drop_copy", "lw_matvec_sequence", "lw_matvec_sequence_workspace_bytes")
 
 _lib = None
 
@@ -74,6 +74,9 @@ def lib() -> ctypes.CDLL:
     L.lw_attn_decode.argtypes = [c_int, vp, vp, vp, vp, i64, i64, i64, i64, ctypes.c_float, vp, i64, vp]
     L.lw_set_attn_variant.restype, L.lw_set_attn_variant.argtypes = c_int, [c_int]
     L.lw_query_attn_variant.restype, L.lw_query_attn_variant.argtypes = c_int, [c_int, i64, i64, i64, i64]
+    L.lw_matvec_sequence_workspace_bytes.restype, L.lw_matvec_sequence_workspace_bytes.argtypes = i64, []
+    L.lw_matvec_sequence.restype = c_int
+    L.lw_matvec_sequence.argtypes = [c_int, c_int, vp, vp, i64, vp]
     L.lw_debug_drop_copy.restype, L.lw_debug_drop_copy.argtypes = c_int, [c_int]
     L.lw_attn_decode_static.restype = c_int
     L.lw_attn_decode_static.argtypes = [c_int, vp, vp, vp, vp, i64, i64, i64, i64, ctypes.c_float, vp]
@@ -155,6 +158,37 @@ def matvec_group(fmt: int, cols: int, items, stream=None) -> None:
         arr[j].W_blocks, arr[j].rows, arr[j].X, arr[j].Y = _addr(w) or None, rows, _addr(x) or None, _addr(y) or None
     _check(lib().lw_matvec_group(fmt, cols, len(items), ctypes.cast(arr, ctypes.c_void_p),
                                  _stream_handle(stream)), "lw_matvec_group")
+
+
+class SeqItem(ctypes.Structure):
+    _fields_ = [("W_blocks", ctypes.c_void_p), ("rows", ctypes.c_int64), ("cols", ctypes.c_int64),
+                ("X", ctypes.c_void_p), ("Y", ctypes.c_void_p), ("flags", ctypes.c_int)]
+
+
+SEQ_DEPENDENT = 1
+
+
+def matvec_sequence_workspace_bytes() -> int:
+    return int(lib().lw_matvec_sequence_workspace_bytes())
+
+
+def seq_items(items):
+    """Marshals (W_blocks, rows, cols, X, Y, flags) tuples into a C array (reusable across calls)."""
+    arr = (SeqItem * len(items))()
+    for j, (w, rows, cols, x, y, flags) in enumerate(items):
+        arr[j].W_blocks, arr[j].rows, arr[j].cols = _addr(w) or None, rows, cols
+        arr[j].X, arr[j].Y, arr[j].flags = _addr(x) or None, _addr(y) or None, flags
+    return arr
+
+
+def matvec_sequence(fmt: int, items, workspace, workspace_bytes: int | None = None, stream=None) -> None:
+    """items: sequence of (W_blocks, rows, cols, X, Y, flags) or an array from seq_items(); one persistent
+    launch for the whole chain (batch 1)."""
+    arr = items if isinstance(items, ctypes.Array) else seq_items(items)
+    if workspace_bytes is None:
+        workspace_bytes = workspace.numel() * workspace.element_size() if hasattr(workspace, "numel") else 0
+    _check(lib().lw_matvec_sequence(fmt, len(arr), ctypes.cast(arr, ctypes.c_void_p), _addr(workspace),
+                                    workspace_bytes, _stream_handle(stream)), "lw_matvec_sequence")
 
 
 def matvec_host(fmt: int, W_blocks, rows: int, cols: int, X_host, Y_host, X_dev, Y_dev,

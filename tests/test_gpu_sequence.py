@@ -1,0 +1,160 @@
+"""GPU parity of lw_matvec_sequence (the persistent kernel that runs a whole chain of mat-vecs in one
+launch) against the fp64 oracle: independent items, phases of several matrices that share their
+activations, chains in which every item reads what the previous one wrote, repeated calls, CUDA-graph
+replay, and the fall-back for shapes the streaming kernels do not take."""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2605_20706_b200 import lw, synth
+
+from gpu_util import Guarded, check_matvec, quantized_weights
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+FMTS = [lw.F16, lw.Q8_0, lw.Q4_0, lw.Q4_K, lw.Q6_K, lw.Q5_K, lw.Q2_K, lw.Q4_1, lw.Q5_0, lw.Q5_1]
+DEP = lw.SEQ_DEPENDENT
+
+
+def _workspace():
+    ws = Guarded(lw.matvec_sequence_workspace_bytes() // 4, fill=None, dtype=torch.int32)
+    return ws
+
+
+def _layer_like(fmt, cols_a, cols_b, seed, scale_rows=1):
+    """A decode-layer-shaped chain: (q, k, v) on x0 | o on x1 | (gate, up) on x2 | down on x3 | ragged extras."""
+    r = scale_rows
+    spec = [("q", 256 * r + 3, cols_a, 0, DEP), ("k", 64 * r + 1, cols_a, 0, 0), ("v", 64 * r, cols_a, 0, 0),
+            ("o", 256 * r, cols_a, 1, DEP), ("gate", 520 * r + 5, cols_a, 2, DEP), ("up", 520 * r + 5, cols_a, 2, 0),
+            ("down", 256 * r + 1, cols_b, 3, DEP), ("tiny", 1, cols_a, 4, DEP), ("small", 37, cols_b, 5, 0),
+            ("tall", 3000 * r + 7, cols_a, 6, DEP)]
+    xs = {}
+    items, keep, refs = [], [], []
+    for j, (name, rows, cols, xid, flags) in enumerate(spec):
+        if xid not in xs:
+            X = synth.activations(seed, xid, 1, cols)
+            xs[xid] = (X, torch.from_numpy(X).cuda())
+        X, xd = xs[xid]
+        blocks = quantized_weights(fmt, rows, cols, seed=seed + j, tensor_id=fmt, outlier_p=0.01)
+        w = torch.from_numpy(blocks).cuda()
+        y = Guarded((1, rows))
+        keep.append((w, xd, y))
+        items.append((w, rows, cols, xd, y.t, flags))
+        refs.append(oracle.matvec(fmt, blocks, rows, cols, X, 1, nthreads=4))
+    return items, keep, refs
+
+
+@pytest.mark.parametrize("fmt", FMTS)
+@pytest.mark.parametrize("cols_a,cols_b", [(4096, 14336), (2048, 8192), (256, 512)])
+def test_sequence_of_layer_shaped_items(fmt, cols_a, cols_b):
+    if fmt == lw.Q6_K and (cols_a % 2048 or cols_b % 2048):
+        cols_a, cols_b = 2048, 6144          # q6_K rows must be whole 16-byte pieces for the streaming kernels
+    if fmt == lw.Q2_K and (cols_a % 1024 or cols_b % 1024):
+        cols_a, cols_b = 1024, 3072
+    items, keep, refs = _layer_like(fmt, cols_a, cols_b, seed=120)
+    ws = _workspace()
+    for _ in range(2):                        # the second call finds the first call's counter value
+        lw.matvec_sequence(fmt, items, ws.t)
+    torch.cuda.synchronize()
+    assert lw.device_status() == 0
+    ws.check("sequence workspace")
+    for (w, x, y), (y_ref, s_ref) in zip(keep, refs):
+        y.check("sequence item")
+        check_matvec(y.t.cpu().numpy(), y_ref, s_ref, "sequence item")
+
+
+@pytest.mark.parametrize("fmt", [lw.Q4_K, lw.Q8_0, lw.F16, lw.Q4_0, lw.Q6_K])
+def test_chain_where_every_item_reads_the_previous_result(fmt):
+    # item i+1's X is item i's Y: the grid-wide barrier before a dependent item is what makes this right.
+    # Each stage is checked against the oracle applied to the GPU's own previous stage (fp32), so errors
+    # do not compound in the comparison.
+    dims = [2048, 4096, 2048, 6144, 2048, 4096, 4096, 2048]       # x0 has dims[0] values; stage i maps dims[i] -> dims[i+1]
+    X0 = synth.activations(130, 0, 1, dims[0])
+    bufs = [torch.from_numpy(X0).cuda()] + [Guarded((1, d)) for d in dims[1:]]
+    mats, items = [], []
+    for i in range(len(dims) - 1):
+        rows, cols = dims[i + 1], dims[i]
+        blocks = quantized_weights(fmt, rows, cols, seed=131 + i, tensor_id=fmt, std=1.0 / np.sqrt(cols))
+        w = torch.from_numpy(blocks).cuda()
+        mats.append((blocks, w, rows, cols))
+        x = bufs[i] if i == 0 else bufs[i].t
+        items.append((w, rows, cols, x, bufs[i + 1].t, DEP))
+    ws = _workspace()
+    arr = lw.seq_items(items)
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        lw.matvec_sequence(fmt, arr, ws.t, stream=side)          # first call outside capture
+    side.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        lw.matvec_sequence(fmt, arr, ws.t, stream=side)
+    for b in bufs[1:]:
+        b.t.fill_(float("nan"))
+    for _ in range(3):
+        graph.replay()
+    torch.cuda.synchronize()
+    assert lw.device_status() == 0
+    x_prev = X0
+    for i, (blocks, w, rows, cols) in enumerate(mats):
+        bufs[i + 1].check("stage %d" % i)
+        got = bufs[i + 1].t.cpu().numpy()
+        y_ref, s_ref = oracle.matvec(fmt, blocks, rows, cols, x_prev, 1, nthreads=8)
+        check_matvec(got, y_ref, s_ref, "chain stage %d" % i)
+        x_prev = got.astype(np.float32)
+
+
+def test_sequence_falls_back_for_shapes_outside_the_streaming_kernels():
+    fmt = lw.Q8_0
+    items, keep, refs = [], [], []
+    for j, (rows, cols) in enumerate([(10, 96), (33, 4096), (5, 32768)]):
+        blocks = quantized_weights(fmt, rows, cols, seed=140 + j)
+        X = synth.activations(140, j, 1, cols)
+        w, x, y = torch.from_numpy(blocks).cuda(), torch.from_numpy(X).cuda(), Guarded((1, rows))
+        keep.append((w, x, y))
+        items.append((w, rows, cols, x, y.t, DEP))
+        refs.append(oracle.matvec(fmt, blocks, rows, cols, X, 1))
+    ws = _workspace()
+    lw.matvec_sequence(fmt, items, ws.t)
+    torch.cuda.synchronize()
+    for (w, x, y), (y_ref, s_ref) in zip(keep, refs):
+        y.check("fallback item")
+        check_matvec(y.t.cpu().numpy(), y_ref, s_ref, "fallback item")
+    # a forced variant takes the same route
+    lw.set_variant(lw.VARIANT_GENERIC)
+    try:
+        items2, keep2, refs2 = _layer_like(lw.Q4_0, 2048, 4096, seed=141)
+        lw.matvec_sequence(lw.Q4_0, items2, ws.t)
+        torch.cuda.synchronize()
+        for (w, x, y), (y_ref, s_ref) in zip(keep2, refs2):
+            check_matvec(y.t.cpu().numpy(), y_ref, s_ref, "forced generic")
+    finally:
+        lw.set_variant(lw.VARIANT_AUTO)
+    assert lw.device_status() == 0
+
+
+def test_sequence_argument_errors_enqueue_nothing():
+    L = lw.lib()
+    w = torch.zeros(4096 * 34 // 32 * 4, dtype=torch.uint8, device="cuda")
+    x = torch.zeros(4096, dtype=torch.float32, device="cuda")
+    y = torch.full((8,), 5.0, dtype=torch.float32, device="cuda")
+    ws = torch.zeros(64, dtype=torch.int32, device="cuda")
+    good = (w, 4, 4096, x, y, 0)
+
+    def call(items, workspace=ws, nbytes=256, fmt=lw.Q8_0):
+        arr = lw.seq_items(items)
+        import ctypes
+        return L.lw_matvec_sequence(fmt, len(items), ctypes.cast(arr, ctypes.c_void_p), lw._addr(workspace), nbytes, None)
+
+    assert call([good], fmt=99) == lw.ERR_FORMAT
+    assert call([good], workspace=None) == lw.ERR_NULL
+    assert call([good], nbytes=8) == lw.ERR_WORKSPACE
+    assert call([good] * 641) == lw.ERR_SHAPE
+    assert call([good, (w, 0, 4096, x, y, 0)]) == lw.ERR_SHAPE
+    assert call([good, (w, 4, 4010, x, y, 0)]) == lw.ERR_SHAPE
+    assert call([good, (w, 4, 4096, None, y, 0)]) == lw.ERR_NULL
+    assert call([good, (w, 4, 4096, x, y, 6)]) == lw.ERR_FORMAT
+    assert call([(w, 4, 4096, lw._addr(x) + 4, y, 0)]) == lw.ERR_ALIGN
+    assert L.lw_matvec_sequence(lw.Q8_0, 1, None, lw._addr(ws), 256, None) == lw.ERR_NULL
+    torch.cuda.synchronize()
+    assert (y == 5.0).all()
