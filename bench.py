@@ -1,14 +1,23 @@
 #!/usr/bin/env python
-"""Decode-step benchmark of the fused dequantize + mat-vec library.
+"""Benchmarks of the fused dequantize + mat-vec library.
 
-One "step" = every mat-vec of one Llama-shaped decode step (7 per layer + lm_head), batch 1 by
-default, issued through the C ABI (`lw_matvec`) on one stream and replayed as a CUDA graph.
-Reports HBM GB/s (algorithmic bytes: weight bytes + 4*batch*(cols+rows) per call, over the step
-time), decode-step-equivalent tokens/s, the roofline fraction against the measured HBM peak, an
-end-to-end number with host<->device copies inside the timed region, and the CPU oracle timed on
-the host cores as a reference baseline.
+Default workload: the decode step.  One "step" = every mat-vec of one Llama-shaped decode step (7 per
+layer + lm_head), batch 1 by default, issued through the C ABI on one stream and replayed as a CUDA
+graph.  Reports HBM GB/s (algorithmic bytes: weight bytes + 4*batch*(cols+rows) per call, over the step
+time), decode-step-equivalent tokens/s, the roofline fraction against the measured HBM peak (and the
+read-only ceiling of the copy pipeline), an end-to-end number through the host-buffer C-ABI call with the
+host<->device copies inside the timed region, and the CPU oracle timed on the host cores as a reference.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--batch B]
+Issue modes of the step (batch 1): `launches` = one lw_matvec_sequence call per step, implemented as one
+grouped launch per phase chained with programmatic dependent launch (LW_SEQ_LAUNCHES, the library's
+default), `persistent` = the same call as one persistent kernel (LW_SEQ_PERSISTENT), `per-call` = one
+lw_matvec per mat-vec.  `auto` (default) times launches and persistent and reports the faster one as the
+headline.
+
+Other workloads: `q8_0_2048` (one 2048x2048 q8_0 mat-vec: hot-L2 latency and a cold figure rotating over
+64 copies), `dequant_<fmt>` (stand-alone dequantisation), `attn*` (decode attention).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--batch B] [--issue MODE]
     python bench.py --impl reference      # times the CPU oracle on a bounded sample
 """
 from __future__ import annotations
@@ -35,6 +44,17 @@ NOMINAL_PEAK_GBS = 8000.0
 FALLBACK_PEAK_GBS = 6650.0
 FMT_ID = {"f16": 0, "q8_0": 1, "q4_0": 2, "q4_K": 3, "q6_K": 4, "q5_K": 5, "q2_K": 6, "q4_1": 7, "q5_0": 8, "q5_1": 9}
 BYTES_PER_WEIGHT = {"f16": 2.0, "q8_0": 34 / 32, "q4_0": 18 / 32, "q4_K": 144 / 256, "q6_K": 210 / 256, "q5_K": 176 / 256, "q2_K": 84 / 256, "q4_1": 20 / 32, "q5_0": 22 / 32, "q5_1": 24 / 32}
+SINGLE_WORKLOADS = ("q8_0_2048",)
+DEQUANT_WORKLOADS = tuple("dequant_" + f for f in FMT_ID)
+
+
+def arithmetic_of(fmt, batch):
+    """What the kernels compute in (the `dtype` key): not a precision claim, the arithmetic that runs."""
+    if fmt == "f16":
+        return "f32 in/out; f16 weights widened, fp32 FMA"
+    if batch == 1:
+        return "f32 in/out; activations as 24-bit block fixed point, int32 dp4a sums, fp32 block scales"
+    return "f32 in/out; batch > 1: per-column passes of the batch-1 kernel (24-bit block fixed point, int32 dp4a) or fp32 FMA tiles"
 
 
 def log(*a):
@@ -123,7 +143,7 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
-# ------------------------------------------------------------------- weight set (host) ---
+# ----------------------------------------------------------------------- common pieces ---
 
 def quantize_tensor(fmt_id, quantize_fn, row_bytes_fn, seed, tensor_id, rows, cols, std, outlier_p, out, pool):
     """Generate tensor `tensor_id` chunk by chunk and quantise it into `out` (uint8 view)."""
@@ -140,31 +160,102 @@ def quantize_tensor(fmt_id, quantize_fn, row_bytes_fn, seed, tensor_id, rows, co
     list(pool.map(job, range(nchunks)))
 
 
-# -------------------------------------------------------------------------- our arm ---
-
-def run_ours(args):
+def device_setup():
     import torch
 
-    from paper_2605_20706_b200 import lw
-
-    from paper_2605_20706_b200 import dist_util
+    from paper_2605_20706_b200 import dist_util, lw
     rank, local_rank, world = dist_util.rank_info()
-    if args.gpus != world and world > 1:
-        log("warning: --gpus %d but WORLD_SIZE %d" % (args.gpus, world))
     if not torch.cuda.is_available():
         raise RuntimeError("bench.py needs a CUDA device (there is no CPU fallback)")
     torch.cuda.set_device(local_rank)
     dist_util.init("nccl", torch.device("cuda", local_rank))
     lw.lib()     # fail loudly here if the extension is missing
+    return torch, dist_util, lw, rank, local_rank, world
 
+
+class Timer:
+    """CUDA-event timing of a callable on the current stream, warm-up first, barrier + synchronize on both sides."""
+
+    def __init__(self, torch, dist_util):
+        self.torch, self.dist = torch, dist_util
+        self.stream = torch.cuda.current_stream()
+
+    def barrier(self):
+        self.torch.cuda.synchronize()
+        self.dist.barrier()
+        self.torch.cuda.synchronize()
+
+    def time(self, fn, steps, warmup):
+        for _ in range(max(3, warmup)):
+            fn()
+        self.barrier()
+        e0, e1 = self.torch.cuda.Event(enable_timing=True), self.torch.cuda.Event(enable_timing=True)
+        e0.record(self.stream)
+        for _ in range(steps):
+            fn()
+        e1.record(self.stream)
+        self.barrier()
+        return e0.elapsed_time(e1) / steps       # ms per call of fn
+
+
+def capture(torch, enqueue, use_graph=True):
+    """Runs `enqueue(stream)` once on a side stream (warm-up outside capture), then captures it into a graph;
+    returns a callable that replays it on the current stream."""
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        enqueue(side)
+    side.synchronize()
+    if not use_graph:
+        cur = torch.cuda.current_stream()
+        return lambda: enqueue(cur)
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        enqueue(side)
+    return graph.replay
+
+
+def read_only_ceiling(lw, timer, buf, nbytes):
+    """GB/s of the streaming kernels' copy pipeline with no arithmetic behind it, over `nbytes` of `buf`."""
+    nbytes -= nbytes % 16
+    if nbytes < (256 << 20):
+        return None
+    ms = timer.time(lambda: lw.probe_read(buf, nbytes), 5, 3)
+    return round(nbytes / (ms * 1e-3) / 1e9, 1)
+
+
+def roofline_block(per_gpu_gbs, kernel, bytes_per_launch, traffic, ceiling=None, bound="hbm"):
+    peak, peak_src = measured_peak()
+    out = {"bound": bound, "achieved": round(per_gpu_gbs, 1), "peak": peak, "peak_source": peak_src, "unit": "GB/s",
+           "frac": round(per_gpu_gbs / peak, 4), "traffic": traffic, "kernel": kernel,
+           "bytes_per_launch_avg": int(bytes_per_launch),
+           "frac_of_nominal_8000": round(per_gpu_gbs / NOMINAL_PEAK_GBS, 4)}
+    if ceiling:
+        out["read_only_ceiling"] = {"value": ceiling, "unit": "GB/s", "frac_of_it": round(per_gpu_gbs / ceiling, 4),
+                                    "what": "lw_probe_read over the workload's weights: the same bulk-copy rings, no arithmetic"}
+    return out
+
+
+# DRAM bytes (read + write) per algorithmic byte of the dominant kernel, from the ncu captures summarised under
+# profiles/ (taken on a few matrices of the workload and scaled by bytes: DRAM traffic of these streaming
+# kernels grows in proportion to the bytes they process).
+TRAFFIC_RATIO = {"llama8b_q4_K": 1.010}
+
+
+# ------------------------------------------------------------------ the decode step ---
+
+def run_step(args):
+    torch, dist_util, lw, rank, local_rank, world = device_setup()
+    if args.gpus != world:
+        log("note: --gpus %d, running with WORLD_SIZE %d" % (args.gpus, world))
     shapes, fmt, std, outlier_p, seed = workload_spec(args.workload, args.layers)
     shapes = filter_shapes(shapes, args.only)
     fmt_id = FMT_ID[fmt]
     batch = args.batch
     ncalls = len(shapes)
     wbytes, abytes = step_bytes(shapes, fmt, batch)
+    timer = Timer(torch, dist_util)
 
-    # ---- build the weight set: every matrix has its own memory (no aliasing between layers)
+    # ---- weights: every matrix has its own memory (no aliasing between layers)
     t0 = time.time()
     offs, total = [], 0
     for _, r, c in shapes:
@@ -211,9 +302,10 @@ def run_ours(args):
 
     lw.set_overlap(not args.no_overlap)
     wptr, xptr, yptr = W.data_ptr(), X.data_ptr(), Y.data_ptr()
+    xhptr, yhptr = X_host.data_ptr(), Y_host.data_ptr()
 
-    # Mat-vecs that are independent in the model (q/k/v share one input, so do gate/up) are issued
-    # on parallel branches; everything else stays in model order on the main branch.
+    # Mat-vecs that are independent in the model (q/k/v share one input, so do gate/up) are issued on parallel
+    # branches in per-call mode; everything else stays in model order on the main branch.
     branch_of = []
     for name, _, _ in shapes:
         leaf = name.split(".")[-1]
@@ -249,8 +341,7 @@ def run_ours(args):
             ev.record(aux[j - 1])
             stream.wait_event(ev)
 
-    # Grouped issue: the same independent mat-vecs (q/k/v, gate/up) go into one lw_matvec_group call
-    # each, everything else is a plain lw_matvec; one branch, model order.
+    # Groups: the independent mat-vecs that share their activations (q/k/v, gate/up); everything else alone.
     groups, i = [], 0
     while i < len(shapes):
         leaf = shapes[i][0].split(".")[-1]
@@ -263,133 +354,126 @@ def run_ours(args):
             groups.append([i])
             i += 1
 
-    def enqueue_grouped(stream):
-        for g in groups:
-            if len(g) == 1:
-                j = g[0]
-                _, r, c = shapes[j]
-                lw.matvec(fmt_id, wptr + offs[j], r, c, xptr + 4 * xoffs[j], yptr + 4 * yoffs[j], batch, stream)
-            else:
-                lw.matvec_group(fmt_id, shapes[g[0]][2],
-                                [(wptr + offs[j], shapes[j][1], xptr + 4 * xoffs[j], yptr + 4 * yoffs[j]) for j in g],
-                                stream)
-
-    # Sequence issue: the whole chain in ONE lw_matvec_sequence call (persistent kernel); q/k/v and
-    # gate/up share their X; every other mat-vec is flagged dependent on what came before it.
+    # Sequence: the whole chain in ONE lw_matvec_sequence call; the members of a group read one X, the first
+    # member of every group is flagged dependent on everything before it.
     seq_list = []
     for g in groups:
         for n, j in enumerate(g):
             _, r, c = shapes[j]
-            x_of = g[0]          # the members of a group read the same activations
-            seq_list.append((wptr + offs[j], r, c, xptr + 4 * xoffs[x_of], yptr + 4 * yoffs[j],
+            seq_list.append((wptr + offs[j], r, c, xptr + 4 * xoffs[g[0]], yptr + 4 * yoffs[j],
                              lw.SEQ_DEPENDENT if n == 0 else 0))
     seq_arr = lw.seq_items(seq_list)
     seq_ws = torch.zeros(lw.matvec_sequence_workspace_bytes() // 4, dtype=torch.int32, device="cuda")
 
-    def enqueue_sequence(stream):
+    def enqueue_launches(stream):
+        lw.set_sequence_mode(lw.SEQ_LAUNCHES)
         lw.matvec_sequence(fmt_id, seq_arr, seq_ws, stream=stream)
 
-    sequence = batch == 1 and args.issue == "sequence"
-    grouped = batch == 1 and args.issue == "grouped"
-    enqueue_step = enqueue_sequence if sequence else (enqueue_grouped if grouped else enqueue_per_call)
-    launches_per_step = 1 if sequence else (len(groups) if grouped else ncalls)
+    def enqueue_persistent(stream):
+        lw.set_sequence_mode(lw.SEQ_PERSISTENT)
+        lw.matvec_sequence(fmt_id, seq_arr, seq_ws, stream=stream)
 
-    side = torch.cuda.Stream()
-    with torch.cuda.stream(side):
-        enqueue_step(side)
-    side.synchronize()
-    if lw.device_status() != 0:
-        raise RuntimeError("device fault recorded during warm-up")
-    graph = None
-    if not args.no_graph:
-        graph = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(graph, stream=side):
-            enqueue_step(side)
+    modes = {"launches": (enqueue_launches, len(groups),
+                          "one lw_matvec_sequence call per step, run as one grouped launch per phase (q/k/v together, "
+                          "gate/up together, the rest alone: %d launches per step) chained with programmatic dependent "
+                          "launch" % len(groups)),
+             "persistent": (enqueue_persistent, 1,
+                            "one lw_matvec_sequence call per step, run as ONE persistent kernel (grid-wide barrier before "
+                            "each dependent mat-vec, weight ring kept filling across boundaries): 1 launch per step"),
+             "per-call": (enqueue_per_call, ncalls, "one lw_matvec call per mat-vec (%d launches per step), q/k/v and "
+                                                    "gate/up on parallel graph branches" % ncalls)}
+    if batch > 1:
+        to_time = ["per-call"]
+    elif args.issue == "auto":
+        to_time = ["launches", "persistent"]
+    else:
+        to_time = [args.issue]
 
-    stream = torch.cuda.current_stream()
-
-    def one_step():
-        if graph is not None:
-            graph.replay()
-        else:
-            enqueue_step(stream)
-
-    def barrier():
+    replays, timings = {}, {}
+    for mode in to_time:
+        replays[mode] = capture(torch, modes[mode][0], not args.no_graph)
         torch.cuda.synchronize()
-        dist_util.barrier()
-        torch.cuda.synchronize()
+        if lw.device_status() != 0:
+            raise RuntimeError("device fault recorded during warm-up (%s)" % mode)
+    # untimed look at every mode, to pick the headline before the clock sampler starts
+    for mode in to_time:
+        timings[mode] = timer.time(replays[mode], max(5, args.steps // 4), args.warmup)
+    headline = min(to_time, key=lambda m: timings[m])
+    one_step = replays[headline]
+    launches_per_step = modes[headline][1]
 
-    # ---- device-resident timing
+    # ---- device-resident timing of the headline mode, clocks sampled during it
     for _ in range(max(3, args.warmup)):
         one_step()
-    barrier()
+    timer.barrier()
     sampler = ClockSampler(local_rank)
     sampler.start()
     time.sleep(0.3)
+    stream = torch.cuda.current_stream()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
+    timer.barrier()
     ev0.record(stream)
     for _ in range(args.steps):
         one_step()
     ev1.record(stream)
-    barrier()
+    timer.barrier()
     ms = ev0.elapsed_time(ev1)
-    # keep the GPU busy a little longer so the clock sampler sees the loaded state
-    t_end = time.time() + 1.0
+    t_end = time.time() + 1.0               # keep the GPU busy a little longer so the sampler sees the loaded state
     while time.time() < t_end:
         one_step()
     torch.cuda.synchronize()
     clocks = sampler.stop()
 
-    # ---- the other issue mode (one call per mat-vec on parallel branches), for comparison
-    other = None
-    if grouped and graph is not None and not args.only:
-        with torch.cuda.stream(side):
-            enqueue_per_call(side)
-        side.synchronize()
-        g2 = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(g2, stream=side):
-            enqueue_per_call(side)
-        for _ in range(3):
-            g2.replay()
-        barrier()
-        o0, o1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        o0.record(stream)
-        for _ in range(args.steps):
-            g2.replay()
-        o1.record(stream)
-        barrier()
-        oms = o0.elapsed_time(o1) / args.steps
-        other = {"issue": "one lw_matvec call per mat-vec (%d launches per step), q/k/v and gate/up on parallel "
-                          "graph branches" % ncalls,
-                 "ms_per_step": round(oms, 5), "value": round((wbytes + abytes) / (oms * 1e-3) / 1e9, 1),
-                 "unit": "GB/s", "tok_per_s": round(1e3 / oms, 2)}
+    def describe(mode, ms_step):
+        return {"issue": modes[mode][2], "ms_per_step": round(ms_step, 5),
+                "value": round((wbytes + abytes) / (ms_step * 1e-3) / 1e9, 1), "unit": "GB/s",
+                "tok_per_s": round(1e3 / ms_step, 2)}
 
-    # ---- end to end: host activations in, host results out, every step
-    for _ in range(3):
-        X.copy_(X_host, non_blocking=True)
-        one_step()
-        Y_host.copy_(Y, non_blocking=True)
-    barrier()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record(stream)
-    for _ in range(args.steps):
-        X.copy_(X_host, non_blocking=True)
-        one_step()
-        Y_host.copy_(Y, non_blocking=True)
-    e1.record(stream)
-    barrier()
-    ms_e2e = e0.elapsed_time(e1)
+    others = {}
+    for mode in to_time:
+        if mode != headline:
+            others[mode] = describe(mode, timer.time(replays[mode], args.steps, 3))
+    if batch == 1 and "per-call" not in to_time and not args.only and not args.no_graph:
+        others["per-call"] = describe("per-call", timer.time(capture(torch, enqueue_per_call), args.steps, 3))
+
+    # ---- end to end through the host-buffer entry points of the C ABI, pinned host memory on both sides, the
+    # copies inside the timed region.  Batch 1: ONE lw_matvec_sequence_host call per step (the step's activation
+    # block in with one copy, the chain in the headline mode, the result block out with one copy).  Beside it
+    # (and alone for batch > 1): one lw_matvec_host call per mat-vec, each with its own two copies.
+    def enqueue_host(stream):
+        for i, (_, r, c) in enumerate(shapes):
+            lw.matvec_host(fmt_id, wptr + offs[i], r, c, xhptr + 4 * xoffs[i], yhptr + 4 * yoffs[i],
+                           xptr + 4 * xoffs[i], yptr + 4 * yoffs[i], batch, stream)
+
+    def enqueue_seq_host(stream):
+        lw.set_sequence_mode(lw.SEQ_PERSISTENT if headline == "persistent" else lw.SEQ_LAUNCHES)
+        lw.matvec_sequence_host(fmt_id, seq_arr, xhptr, xptr, 4 * xt, yptr, yhptr, 4 * yt, seq_ws, stream=stream)
+
+    ms_percall_host = timer.time(capture(torch, enqueue_host, not args.no_graph), max(3, args.steps // 5), 3)
+    if batch == 1:
+        ms_host = timer.time(capture(torch, enqueue_seq_host, not args.no_graph), args.steps, 3) * args.steps
+        h2d, d2h = 4 * xt, 4 * yt
+        e2e_path = "one lw_matvec_sequence_host call per step: the step's %d-byte activation block from pinned host " \
+                   "memory to the device in one copy, the chain (%s), the %d-byte result block back in one copy" % (
+                       4 * xt, headline, 4 * yt)
+    else:
+        ms_host = ms_percall_host * args.steps
+        h2d = sum(4 * batch * c for _, _, c in shapes)
+        d2h = sum(4 * batch * r for _, r, _ in shapes)
+        e2e_path = "one lw_matvec_host call per mat-vec"
+    lw.set_sequence_mode(lw.SEQ_AUTO)
     if lw.device_status() != 0:
         raise RuntimeError("device fault recorded during the timed region")
 
-    ms, ms_e2e = dist_util.max_over_ranks([ms, ms_e2e], device="cuda")
+    ceiling = read_only_ceiling(lw, timer, W, total) if not args.only else None
+    ms, ms_host = dist_util.max_over_ranks([ms, ms_host], device="cuda")
 
     step_ms = ms / args.steps
     total_bytes = (wbytes + abytes) * world
     gbs = total_bytes / (step_ms * 1e-3) / 1e9
-    peak, peak_src = measured_peak()
     per_gpu_gbs = gbs / world
+    kernel = ("matvec_seq_kernel" if headline == "persistent" else "matvec_stream_kernel") + \
+        "<%s%s>" % ("Idot_" if fmt != "f16" else "", fmt)
     result = {
         "metric": METRIC,
         "value": round(gbs, 1),
@@ -401,19 +485,14 @@ def run_ours(args):
         "higher_is_better": True,
         "scaling": "weak",
         "vs_baseline": None,
-        "dtype": "f32",
+        "dtype": arithmetic_of(fmt, batch),
         "data": "synthetic",
         "config": {
-            "workload": "%s: %d mat-vecs per decode step, batch %d, weights %.3f GB in %s, "
-                        "fp32 activations; %s%s%s" % (
-                            args.workload, ncalls, batch, wbytes / 1e9, fmt,
-                            ("lw_matvec_group for q/k/v and for gate/up (independent in the model), lw_matvec for "
-                             "the rest: %d launches per step" % launches_per_step) if grouped
-                            else "one lw_matvec call per mat-vec",
-                            ", replayed as one CUDA graph" if graph is not None else "",
-                            (", programmatic dependent launch between calls" if not args.no_overlap else "") +
-                            ("" if (args.serial or grouped) else "; q/k/v and gate/up (independent in the model) on parallel graph branches")),
-            "format": fmt, "batch": batch, "calls_per_step": ncalls,
+            "workload": "%s: %d mat-vecs per decode step, batch %d, weights %.3f GB in %s, fp32 activations; %s%s%s" % (
+                args.workload, ncalls, batch, wbytes / 1e9, fmt, modes[headline][2],
+                "" if args.no_graph else ", replayed as one CUDA graph",
+                "" if (args.no_overlap or headline != "per-call") else ", programmatic dependent launch between calls"),
+            "format": fmt, "batch": batch, "calls_per_step": ncalls, "issue": headline,
             "weight_bytes": wbytes, "activation_bytes": abytes,
             "l2": "weight set is %.0fx the 126 MB L2 and is streamed evict-first; no flush needed" % (wbytes / 126e6),
             "parallelism": "replicas only (one independent decode step per GPU)" if world > 1 else "single GPU",
@@ -423,28 +502,37 @@ def run_ours(args):
         "effective_gflops": round(world * sum(2.0 * r * c * batch for _, r, c in shapes) / (step_ms * 1e-3) / 1e9, 1),
         "clocks": clocks,
         "gpu_launches": args.steps * launches_per_step,
-        "per_call": other,
+        "other_issue_modes": others,
         "e2e": {
-            "value": round((wbytes + abytes) * world / (ms_e2e / args.steps * 1e-3) / 1e9, 1),
+            "value": round((wbytes + abytes) * world / (ms_host / args.steps * 1e-3) / 1e9, 1),
             "unit": "GB/s",
-            "ms_per_step": round(ms_e2e / args.steps, 5),
-            "tok_per_s": round(world * args.steps * 1e3 / ms_e2e, 2),
-            "h2d_bytes_per_step": int(X_host.numel() * 4),
-            "d2h_bytes_per_step": int(Y_host.numel() * 4),
+            "ms_per_step": round(ms_host / args.steps, 5),
+            "tok_per_s": round(world * args.steps * 1e3 / ms_host, 2),
+            "h2d_bytes_per_step": int(h2d),
+            "d2h_bytes_per_step": int(d2h),
+            "path": e2e_path + ("" if args.no_graph else ", replayed as one CUDA graph"),
+            "per_matvec_host_calls": {
+                "what": "one lw_matvec_host call per mat-vec (%d calls, each: pinned host X -> device, kernel, Y -> pinned "
+                        "host): %d small copies per step, bound by copy-engine latency" % (ncalls, 2 * ncalls),
+                "ms_per_step": round(ms_percall_host, 5),
+                "value": round((wbytes + abytes) / (ms_percall_host * 1e-3) / 1e9, 1), "unit": "GB/s",
+                "h2d_bytes_per_step": int(sum(4 * batch * c for _, _, c in shapes)),
+                "d2h_bytes_per_step": int(sum(4 * batch * r for _, r, _ in shapes))},
         },
-        "roofline": {
-            "bound": "hbm",
-            "achieved": round(per_gpu_gbs, 1),
-            "peak": peak,
-            "peak_source": peak_src,
-            "unit": "GB/s",
-            "frac": round(per_gpu_gbs / peak, 4),
-            "traffic": (int(TRAFFIC_RATIO[args.workload] * (wbytes + abytes) / launches_per_step)
-                        if args.workload in TRAFFIC_RATIO and batch == 1 else None),
-            "kernel": "matvec_stream_kernel<%s%s>" % ("Idot_" if fmt != "f16" and batch == 1 else "", fmt),
-            "bytes_per_launch_avg": int((wbytes + abytes) / launches_per_step),
-        },
+        "roofline": roofline_block(
+            per_gpu_gbs, kernel, (wbytes + abytes) / launches_per_step,
+            int(TRAFFIC_RATIO[args.workload] * (wbytes + abytes) / launches_per_step)
+            if args.workload in TRAFFIC_RATIO and batch == 1 else None, ceiling),
     }
+    if batch > 1:
+        # the binding bound from batch 2 on is instruction issue, not HBM: state it with its derivation
+        flops = sum(2.0 * r * c * batch for _, r, c in shapes)
+        alu_peak = 148 * 128 * 1.965e9 * 2 / 1e12
+        result["roofline_alu"] = {
+            "bound": "alu", "achieved": round(flops / (step_ms * 1e-3) / 1e12, 2), "peak": round(alu_peak, 1),
+            "unit": "TFLOP/s", "frac": round(flops / (step_ms * 1e-3) / 1e12 / alu_peak, 4),
+            "derivation": "148 SMs x 128 fp32 lanes x 1.965 GHz x 2 flop per FMA = 74.4 TFLOP/s of plain FMA issue; "
+                          "the integer-dot form needs 3 dp4a per 4 weight-columns on a half-rate pipe (about 50)"}
 
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         result["cpu_baseline"] = cpu_baseline_leg(shapes, fmt, fmt_id, batch, seed, std, outlier_p, keep_host, xh,
@@ -454,19 +542,13 @@ def run_ours(args):
     dist_util.shutdown()
 
 
-# Measured DRAM bytes (read + write) per algorithmic byte of the dominant kernel, from the ncu capture
-# summarised under profiles/ (taken on two matrices of the workload and scaled by bytes, since DRAM
-# traffic of this streaming kernel grows in proportion to the bytes it processes).
-TRAFFIC_RATIO = {"llama8b_q4_K": 1.010}
-
-
 # --------------------------------------------------------- oracle legs (CPU, rank 0) ---
 
 def cpu_baseline_leg(shapes, fmt, fmt_id, batch, seed, std, outlier_p, keep_host, xh, xoffs, Y_dev, yoffs,
                      seconds):
     """Times the oracle (as it stands) on a bounded sample of the step -- whole matrices, regenerated
-    from the seeded recipe and quantised by the oracle's own quantiser -- and checks the GPU results
-    of those matrices against it with the mat-vec tolerance."""
+    from the seeded recipe and quantised by the oracle's own quantiser -- once on all cores and once
+    single-threaded, and checks the GPU results of those matrices against it with the mat-vec tolerance."""
     import oracle
     cores = os.cpu_count() or 1
     total_w = sum(r * c for _, r, c in shapes)
@@ -485,6 +567,7 @@ def cpu_baseline_leg(shapes, fmt, fmt_id, batch, seed, std, outlier_p, keep_host
     order += [i for i in range(7, len(shapes) - 1)]
     y_gpu = Y_dev.cpu().numpy()
     worst, cpu_time, nbytes, used, chosen, bytes_equal = 0.0, 0.0, 0, 0, [], True
+    single_time, single_bytes, single_w = 0.0, 0, 0
     t_leg = time.time()
     for i in order:
         _, r, c = shapes[i]
@@ -504,6 +587,13 @@ def cpu_baseline_leg(shapes, fmt, fmt_id, batch, seed, std, outlier_p, keep_host
         chosen.append(i)
         got = y_gpu[yoffs[i]:yoffs[i] + batch * r].reshape(batch, r).astype(np.float64)
         worst = max(worst, float((np.abs(got - y_ref) / (1e-4 * s_ref + 1e-6)).max()))
+        if single_time < seconds / 2:           # single-threaded: the first rows of the same matrix
+            rr = max(1, min(r, int(2.0e7 // c)))
+            t = time.time()
+            oracle.matvec(fmt_id, blocks[:oracle.row_bytes(fmt_id, c) * rr], rr, c, x, batch, nthreads=1)
+            single_time += time.time() - t
+            single_bytes += int(rr * c * BYTES_PER_WEIGHT[fmt]) + 4 * batch * (rr + c)
+            single_w += rr * c
     pool.shutdown()
     return {
         "value": round(nbytes / cpu_time / 1e9, 4),
@@ -514,6 +604,10 @@ def cpu_baseline_leg(shapes, fmt, fmt_id, batch, seed, std, outlier_p, keep_host
                   "%.1f%% of the step's weights), every row; %.1f s of oracle mat-vec time" % (
                       len(chosen), len(shapes), 100.0 * used / total_w, cpu_time),
         "tok_per_s_equiv": round(1.0 / (cpu_time * total_w / used), 5),
+        "single_thread": {"value": round(single_bytes / max(single_time, 1e-9) / 1e9, 4), "unit": "GB/s", "cores": 1,
+                          "sample": "the first rows (up to 2e7 weights) of the first of those matrices, %.2f%% of the "
+                                    "step's weights, %.1f s" % (100.0 * single_w / total_w, single_time),
+                          "tok_per_s_equiv": round(1.0 / (max(single_time, 1e-9) * total_w / max(single_w, 1)), 6)},
         "gpu_vs_oracle_worst_err_over_tol": round(worst, 4),
         "parity_ok": bool(worst <= 1.0),
         "host_quantiser_bytes_equal_oracle": bytes_equal,
@@ -545,6 +639,16 @@ def run_reference(args):
         for blocks, rr, c, x in mats:
             oracle.matvec(fmt_id, blocks, rr, c, x, batch, nthreads=cores)
 
+    reference_line(args, METRIC, step, nbytes,
+                   "first %d rows of each of the first layer's 7 matrices (%d weights = %.3f%% of a step) per step" % (
+                       args.ref_rows, nweights, 100.0 * nweights / sum(r * c for _, r, c in shapes)),
+                   {"format": fmt, "batch": batch},
+                   extra={"tok_per_s_fraction": nweights / sum(r * c for _, r, c in shapes)})
+
+
+def reference_line(args, metric, step, nbytes, sample_txt, config_extra, extra=None):
+    """Times `step` (the oracle on a bounded sample) and prints the reference arm's JSON line."""
+    cores = os.cpu_count() or 1
     for _ in range(max(1, args.warmup)):
         step()
     t = time.time()
@@ -552,23 +656,258 @@ def run_reference(args):
         step()
     dt = (time.time() - t) / args.steps
     gbs = nbytes / dt / 1e9
-    total_w = sum(r * c for _, r, c in shapes)
-    sample_txt = ("first %d rows of each of the first layer's 7 matrices (%d weights = %.3f%% of a step) per "
-                  "step" % (args.ref_rows, nweights, 100.0 * nweights / total_w))
-    print(json.dumps({
-        "impl": "reference",
-        "metric": METRIC, "value": round(gbs, 4), "unit": "GB/s",
+    line = {
+        "impl": "reference", "metric": metric, "value": round(gbs, 4), "unit": "GB/s",
         "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": args.steps, "warmup": max(1, args.warmup),
         "ms_per_step": round(dt * 1e3, 3), "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f64", "data": "synthetic",
-        "config": {"workload": "%s (CPU oracle on a bounded sample: %s)" % (args.workload, sample_txt),
-                   "format": fmt, "batch": batch},
-        "tok_per_s": round(nweights / total_w / dt, 5),
+        "config": dict({"workload": "%s (CPU oracle on a bounded sample: %s)" % (args.workload, sample_txt)}, **config_extra),
         "cpu_baseline": {"value": round(gbs, 4), "unit": "GB/s", "cores": cores, "kind": "oracle", "sample": sample_txt},
         "e2e": {"value": round(gbs, 4), "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
-    }), flush=True)
+    }
+    if extra and "tok_per_s_fraction" in extra:
+        line["tok_per_s"] = round(extra["tok_per_s_fraction"] / dt, 5)
+    print(json.dumps(line), flush=True)
 
+
+# ------------------------------------------- one small mat-vec: hot and cold (config 1) ---
+
+SINGLE_METRIC = "single mat-vec (q8_0 2048x2048, batch 1): HBM GB/s cold, microseconds per call hot and cold"
+
+
+def single_spec():
+    return FMT_ID["q8_0"], 2048, 2048, 64, 1       # format, rows, cols, copies, seed
+
+
+def run_single(args):
+    """Config 1: W 2048x2048 q8_0, x 2048.  Launch-latency-bound by construction (4.46 MB per call), so two figures:
+    hot = the same matrix again and again (L2-resident), cold = rotating over 64 copies (285 MB, 2.3x the L2)."""
+    torch, dist_util, lw, rank, local_rank, world = device_setup()
+    fmt_id, rows, cols, copies, seed = single_spec()
+    timer = Timer(torch, dist_util)
+    w32 = synth.weights(seed, 0, rows, cols, 0.02, 0.0)
+    blocks = lw.quantize(fmt_id, w32)
+    nb = blocks.size
+    stride = (nb + 255) & ~255
+    W = torch.empty(copies * stride, dtype=torch.uint8, device="cuda")
+    for k in range(copies):
+        W[k * stride:k * stride + nb].copy_(torch.from_numpy(blocks))
+    x_np = synth.activations(seed, 0, 1, cols)
+    X_host = torch.from_numpy(x_np.copy()).pin_memory()
+    Y_host = torch.empty(copies, rows, dtype=torch.float32).pin_memory()
+    X = X_host.cuda()
+    Y = torch.zeros(copies, rows, dtype=torch.float32, device="cuda")
+    lw.set_overlap(not args.no_overlap)
+    wp, xp, yp = W.data_ptr(), X.data_ptr(), Y.data_ptr()
+
+    def enqueue_cold(stream):
+        for k in range(copies):
+            lw.matvec(fmt_id, wp + k * stride, rows, cols, xp, yp + 4 * rows * k, 1, stream)
+
+    def enqueue_hot(stream):
+        for k in range(copies):
+            lw.matvec(fmt_id, wp, rows, cols, xp, yp, 1, stream)
+
+    seq = lw.seq_items([(wp + k * stride, rows, cols, xp, yp + 4 * rows * k, lw.SEQ_DEPENDENT) for k in range(copies)])
+    seq_ws = torch.zeros(64, dtype=torch.int32, device="cuda")
+
+    def enqueue_seq(stream):
+        lw.set_sequence_mode(lw.SEQ_PERSISTENT)
+        lw.matvec_sequence(fmt_id, seq, seq_ws, stream=stream)
+        lw.set_sequence_mode(lw.SEQ_AUTO)
+
+    def enqueue_host(stream):
+        for k in range(copies):
+            lw.matvec_host(fmt_id, wp + k * stride, rows, cols, X_host.data_ptr(), Y_host.data_ptr() + 4 * rows * k,
+                           xp, yp + 4 * rows * k, 1, stream)
+
+    cold, hot, seqr, host = (capture(torch, f, not args.no_graph) for f in (enqueue_cold, enqueue_hot, enqueue_seq, enqueue_host))
+    # parity of every copy's result against the oracle before timing
+    parity = None
+    if rank == 0 and not args.no_cpu_baseline:
+        import oracle
+        cold()
+        torch.cuda.synchronize()
+        y_ref, s_ref = oracle.matvec(fmt_id, oracle.quantize(fmt_id, w32), rows, cols, x_np, 1, nthreads=os.cpu_count() or 1)
+        got = Y.cpu().numpy().astype(np.float64)
+        parity = float((np.abs(got - y_ref) / (1e-4 * s_ref + 1e-6)).max())
+        if not parity <= 1.0:
+            raise RuntimeError("parity check failed: worst error / tolerance = %.3g" % parity)
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    time.sleep(0.3)
+    ms_cold = timer.time(cold, args.steps, args.warmup)
+    ms_hot = timer.time(hot, args.steps, args.warmup)
+    ms_seq = timer.time(seqr, args.steps, args.warmup)
+    ms_host = timer.time(host, args.steps, 3)
+    t_end = time.time() + 0.7
+    while time.time() < t_end:
+        cold()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    if lw.device_status() != 0:
+        raise RuntimeError("device fault recorded during the timed region")
+    ms_cold, ms_hot, ms_seq, ms_host = dist_util.max_over_ranks([ms_cold, ms_hot, ms_seq, ms_host], device="cuda")
+    call_bytes = nb + 4 * (rows + cols)
+    step_b = copies * call_bytes
+    gbs = world * step_b / (ms_cold * 1e-3) / 1e9
+    result = {
+        "metric": SINGLE_METRIC, "value": round(gbs, 1), "unit": "GB/s", "n_gpus": world, "steps": args.steps,
+        "warmup": max(3, args.warmup), "ms_per_step": round(ms_cold, 5), "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": arithmetic_of("q8_0", 1), "data": "synthetic",
+        "config": {"workload": "q8_0_2048: one step = %d lw_matvec calls, one per copy of a 2048x2048 q8_0 matrix "
+                               "(4,456,448 bytes each; %d copies = %.0f MB, %.1fx the 126 MB L2, so every call reads cold "
+                               "weights), batch 1, consecutive calls on one stream with programmatic dependent launch%s" % (
+                                   copies, copies, copies * nb / 1e6, copies * nb / 126e6,
+                                   "" if args.no_graph else ", replayed as one CUDA graph"),
+                   "format": "q8_0", "batch": 1, "calls_per_step": copies, "weight_bytes": copies * nb,
+                   "l2": "rotation over %d copies (%.1fx the L2)" % (copies, copies * nb / 126e6)},
+        "us_per_call_cold": round(1e3 * ms_cold / copies, 3),
+        "us_per_call_hot_l2": round(1e3 * ms_hot / copies, 3),
+        "hot_l2": {"what": "the same matrix %d times in a row (L2-resident after the first call)" % copies,
+                   "value": round(step_b / (ms_hot * 1e-3) / 1e9, 1), "unit": "GB/s of algorithmic bytes (served by L2)"},
+        "sequence": {"what": "the same %d cold calls as ONE persistent lw_matvec_sequence kernel (each item dependent on the previous one)" % copies,
+                     "us_per_call": round(1e3 * ms_seq / copies, 3), "value": round(step_b / (ms_seq * 1e-3) / 1e9, 1),
+                     "unit": "GB/s"},
+        "floor_us_per_call": {"at_measured_peak": round(call_bytes / measured_peak()[0] / 1e3, 3),
+                              "at_nominal_8000": round(call_bytes / 8000.0 / 1e3, 3)},
+        "clocks": clocks, "gpu_launches": args.steps * copies,
+        "parity_worst_error_over_tolerance": None if parity is None else round(parity, 4),
+        "e2e": {"value": round(world * step_b / (ms_host * 1e-3) / 1e9, 1), "unit": "GB/s",
+                "ms_per_step": round(ms_host, 5), "us_per_call": round(1e3 * ms_host / copies, 3),
+                "h2d_bytes_per_step": copies * 4 * cols, "d2h_bytes_per_step": copies * 4 * rows,
+                "path": "one lw_matvec_host call per mat-vec (pinned host X in, pinned host Y out)"},
+        "roofline": roofline_block(gbs / world, "matvec_stream_kernel<Idot_q8_0>", call_bytes, None),
+    }
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import oracle
+        ob = oracle.quantize(fmt_id, w32)
+        cores = os.cpu_count() or 1
+        leg = {}
+        for name, nthr in (("all_cores", cores), ("single_thread", 1)):
+            reps, t = 0, time.time()
+            while reps < 1 or time.time() - t < args.cpu_seconds / 2:
+                oracle.matvec(fmt_id, ob, rows, cols, x_np, 1, nthreads=nthr)
+                reps += 1
+            dt = (time.time() - t) / reps
+            leg[name] = {"value": round(call_bytes / dt / 1e9, 4), "unit": "GB/s", "cores": nthr,
+                         "us_per_call": round(dt * 1e6, 1), "repetitions": reps}
+        result["cpu_baseline"] = {"value": leg["all_cores"]["value"], "unit": "GB/s", "cores": cores, "kind": "oracle",
+                                  "sample": "the whole 2048x2048 mat-vec, %d repetitions" % leg["all_cores"]["repetitions"],
+                                  "us_per_call": leg["all_cores"]["us_per_call"], "single_thread": leg["single_thread"]}
+    if rank == 0:
+        print(json.dumps(result), flush=True)
+    dist_util.shutdown()
+
+
+def run_single_reference(args):
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    import oracle
+    fmt_id, rows, cols, copies, seed = single_spec()
+    ob = oracle.quantize(fmt_id, synth.weights(seed, 0, rows, cols, 0.02, 0.0))
+    x = synth.activations(seed, 0, 1, cols)
+    cores = os.cpu_count() or 1
+    reference_line(args, SINGLE_METRIC, lambda: oracle.matvec(fmt_id, ob, rows, cols, x, 1, nthreads=cores),
+                   ob.size + 4 * (rows + cols), "one 2048x2048 q8_0 mat-vec per step (1 of the GPU arm's %d calls per step)" % copies,
+                   {"format": "q8_0", "batch": 1})
+
+
+# ------------------------------------------------------------ stand-alone dequantisation ---
+
+DEQUANT_METRIC = "stand-alone dequantisation: HBM GB/s of (block bytes read + 4 bytes written) per weight"
+DEQUANT_WEIGHTS = 1 << 28
+
+
+def run_dequant(args):
+    """One step = one lw_dequant call over 2^28 weights (1 GiB of fp32 out, 8x the L2)."""
+    torch, dist_util, lw, rank, local_rank, world = device_setup()
+    fmt = args.workload[len("dequant_"):]
+    fmt_id = FMT_ID[fmt]
+    n = DEQUANT_WEIGHTS
+    timer = Timer(torch, dist_util)
+    nb = lw.row_bytes(fmt_id, n)
+    # blocks: a seeded 16 Mi-weight tile quantised on the host and repeated (timing depends on bytes, not values)
+    tile_n = 1 << 24
+    tile = lw.quantize(fmt_id, synth.normal(77, fmt_id, tile_n, 0.02, 0.01))
+    W_host = torch.from_numpy(np.tile(tile, n // tile_n)).pin_memory()
+    W = W_host.cuda()
+    out = torch.empty(n, dtype=torch.float32, device="cuda")
+    out_host = torch.empty(n, dtype=torch.float32).pin_memory()
+    step = lambda: lw.dequant(fmt_id, W, n, out)
+    step()
+    torch.cuda.synchronize()
+    parity = None
+    if rank == 0 and not args.no_cpu_baseline:
+        import oracle
+        m = 1 << 20
+        want = oracle.dequant(fmt_id, oracle.quantize(fmt_id, synth.normal(77, fmt_id, tile_n, 0.02, 0.01))[:oracle.row_bytes(fmt_id, m)], m)
+        for start in (0, n - tile_n):                 # first and last tile: the first 2^20 weights of each, bit for bit
+            got = out[start:start + m].cpu().numpy()
+            if not (got.view(np.uint32) == want.view(np.uint32)).all():
+                raise RuntimeError("dequant parity failed at %d" % start)
+        parity = True
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    time.sleep(0.3)
+    ms = timer.time(step, args.steps, args.warmup)
+    t_end = time.time() + 0.7
+    while time.time() < t_end:
+        step()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+
+    def e2e_step():
+        W.copy_(W_host, non_blocking=True)
+        step()
+        out_host.copy_(out, non_blocking=True)
+
+    ms_e2e = timer.time(e2e_step, max(2, args.steps // 10), 3)
+    ms, ms_e2e = dist_util.max_over_ranks([ms, ms_e2e], device="cuda")
+    step_b = nb + 4 * n
+    gbs = world * step_b / (ms * 1e-3) / 1e9
+    result = {
+        "metric": DEQUANT_METRIC, "value": round(gbs, 1), "unit": "GB/s", "n_gpus": world, "steps": args.steps,
+        "warmup": max(3, args.warmup), "ms_per_step": round(ms, 5), "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bytes -> f32, bit-exact decode", "data": "synthetic",
+        "config": {"workload": "%s: one lw_dequant call over 2^28 weights per step (%.3f GB of %s blocks in, 1.074 GB of "
+                               "fp32 out; the output alone is 8.5x the 126 MB L2)" % (args.workload, nb / 1e9, fmt),
+                   "format": fmt, "weights": n, "bytes_per_weight": BYTES_PER_WEIGHT[fmt] + 4,
+                   "l2": "input + output are %.1fx the L2; streaming stores" % (step_b / 126e6)},
+        "weights_per_s": round(world * n / (ms * 1e-3), 1), "clocks": clocks, "gpu_launches": args.steps,
+        "parity_bit_exact_on_samples": parity,
+        "e2e": {"value": round(world * step_b / (ms_e2e * 1e-3) / 1e9, 1), "unit": "GB/s", "ms_per_step": round(ms_e2e, 4),
+                "h2d_bytes_per_step": int(nb), "d2h_bytes_per_step": int(4 * n),
+                "path": "blocks from pinned host memory in, lw_dequant, fp32 result back to pinned host memory (PCIe-bound)"},
+        "roofline": roofline_block(gbs / world, "dequant_kernel<%s>" % fmt, step_b, None),
+    }
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        import oracle
+        m = 1 << 22
+        ob = oracle.quantize(fmt_id, synth.normal(77, fmt_id, m, 0.02, 0.01))
+        reps, t = 0, time.time()
+        while reps < 1 or time.time() - t < args.cpu_seconds:
+            oracle.dequant(fmt_id, ob, m)
+            reps += 1
+        dt = (time.time() - t) / reps
+        result["cpu_baseline"] = {"value": round((ob.size + 4 * m) / dt / 1e9, 4), "unit": "GB/s", "cores": 1, "kind": "oracle",
+                                  "sample": "2^22 weights (1.6%% of a step) per repetition, %d repetitions" % reps}
+    if rank == 0:
+        print(json.dumps(result), flush=True)
+    dist_util.shutdown()
+
+
+def run_dequant_reference(args):
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    import oracle
+    fmt = args.workload[len("dequant_"):]
+    fmt_id = FMT_ID[fmt]
+    m = 1 << 22
+    ob = oracle.quantize(fmt_id, synth.normal(77, fmt_id, m, 0.02, 0.01))
+    reference_line(args, DEQUANT_METRIC, lambda: oracle.dequant(fmt_id, ob, m), ob.size + 4 * m,
+                   "2^22 weights (1.6% of the GPU arm's step) per step", {"format": fmt})
 
 
 # ------------------------------------------------------------- decode attention workloads ---
@@ -787,6 +1126,17 @@ def run_attn_reference(args):
     }), flush=True)
 
 
+def spawn_ranks(args):
+    """`python bench.py --gpus N` without a torchrun environment: start the N ranks here (one per GPU)."""
+    import socket
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(args.gpus),
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    raise SystemExit(subprocess.call(cmd))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -794,26 +1144,30 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama8b_q4_K",
-                    choices=sorted(synth.WORKLOADS) + sorted(synth.ATTN_WORKLOADS))
+                    choices=sorted(synth.WORKLOADS) + sorted(synth.ATTN_WORKLOADS) + list(SINGLE_WORKLOADS) +
+                    list(DEQUANT_WORKLOADS))
     ap.add_argument("--batch", type=int, default=1)
     ap.add_argument("--layers", type=int, default=None, help="use fewer layers (debugging only)")
     ap.add_argument("--only", default=None, help="comma-separated substrings: keep only matching mat-vecs "
                                                   "(profiling of single kernels)")
+    ap.add_argument("--issue", default="auto", choices=["auto", "launches", "persistent", "per-call"],
+                    help="how the step's mat-vecs are issued at batch 1 (auto: time launches and persistent, report the faster)")
     ap.add_argument("--no-graph", action="store_true")
-    ap.add_argument("--issue", default="sequence", choices=["sequence", "grouped", "per-call"],
-                    help="sequence: one lw_matvec_sequence call per step; grouped: lw_matvec_group for q/k/v and "
-                         "gate/up, lw_matvec for the rest; per-call: one lw_matvec per mat-vec")
-    ap.add_argument("--serial", action="store_true", help="one branch: every mat-vec waits for the previous one")
+    ap.add_argument("--serial", action="store_true", help="per-call mode on one branch: every mat-vec waits for the previous one")
     ap.add_argument("--no-overlap", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=4.0)
     ap.add_argument("--ref-rows", type=int, default=512)
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl == "ours":
+        spawn_ranks(args)
     attn = args.workload in synth.ATTN_WORKLOADS
+    single = args.workload in SINGLE_WORKLOADS
+    deq = args.workload in DEQUANT_WORKLOADS
     if args.impl == "reference":
-        (run_attn_reference if attn else run_reference)(args)
+        (run_attn_reference if attn else run_single_reference if single else run_dequant_reference if deq else run_reference)(args)
     else:
-        (run_attn if attn else run_ours)(args)
+        (run_attn if attn else run_single if single else run_dequant if deq else run_step)(args)
 
 
 if __name__ == "__main__":

@@ -152,25 +152,29 @@ typedef struct {
 } lw_group_item;
 int lw_matvec_group(int fmt, int64_t cols, int n_items, const lw_group_item* items, void* stream);
 
-/* A whole chain of batch-1 mat-vecs of one format in ONE launch [Sec 3.1, 3.2: the runtime groups operations
+/* A whole chain of batch-1 mat-vecs of one format in ONE call [Sec 3.1, 3.2: the runtime groups operations
  * into compute passes; the whole mat-vec chain of a decode step is one pass here].  The items run in the
  * order given.  Consecutive items that read the same X (same pointer, same cols) and are not flagged
  * dependent form one phase whose rows are shared out over all SMs together (q/k/v, gate/up).  An item
  * flagged LW_SEQ_DEPENDENT reads (X) or overwrites (Y) memory that an earlier item of the sequence writes
- * or reads: before it starts, every earlier item has finished device-wide (a grid-wide barrier inside the
- * kernel).  Without the flag an item may run concurrently with its predecessors.  The kernel is persistent,
- * one CTA per SM, launched cooperatively: the weight ring keeps filling across item boundaries (weights are
- * constant data), so a boundary costs a barrier and the activation fetch instead of a kernel launch with a
- * cold pipeline.
+ * or reads: before it starts, every earlier item has finished device-wide.  Without the flag an item may
+ * run concurrently with its predecessors.  Two implementations (lw_set_sequence_mode):
+ *   LW_SEQ_LAUNCHES   one grouped launch per phase, chained with programmatic dependent launch (a kernel's
+ *                     CTAs are placed and set up while its predecessor finishes and wait for it before they
+ *                     touch W or X); the default (LW_SEQ_AUTO) because it measures faster on B200;
+ *   LW_SEQ_PERSISTENT one persistent kernel, one CTA per SM, launched cooperatively, with a grid-wide barrier
+ *                     before each dependent item; the weight ring keeps filling across item boundaries
+ *                     (weights are constant data), so a boundary costs a barrier and the activation fetch
+ *                     instead of a launch with a cold pipeline.
  * Each item is what lw_matvec takes at batch 1 (W: rows * lw_row_bytes(fmt, cols) bytes; X: cols floats;
  * Y: rows floats; all device, 16-byte aligned); n_items <= 640, at most 320 phases.
  * workspace: device, at least lw_matvec_sequence_workspace_bytes() bytes, 16-byte aligned, owned by the
  *           caller, need not be initialised (the call clears what it needs on `stream` first); sequences that
  *           may run concurrently need separate workspaces.
  * `items` is host memory, read during the call only.  Results and accuracy are those of lw_matvec.
- * When a shape is not covered by the streaming kernels, a variant is forced, or the device cannot launch
- * cooperatively, the items are issued one after the other with lw_matvec on `stream` (stream order then
- * provides every dependency).  Asynchronous on `stream`; can be captured into a CUDA graph.
+ * When a shape is not covered by the streaming kernels or a variant is forced, the items are issued one
+ * after the other with lw_matvec on `stream` (stream order then provides every dependency); a device that
+ * cannot launch cooperatively gets LW_SEQ_LAUNCHES.  Asynchronous on `stream`; can be captured into a CUDA graph.
  * Errors: as lw_matvec per item, LW_ERR_SHAPE for n_items outside 1..640, LW_ERR_WORKSPACE. */
 typedef struct {
     const void* W_blocks;
@@ -184,6 +188,19 @@ enum { LW_SEQ_DEPENDENT = 1 };
 int64_t lw_matvec_sequence_workspace_bytes(void);
 int lw_matvec_sequence(int fmt, int n_items, const lw_seq_item* items, void* workspace, int64_t workspace_bytes,
                        void* stream);
+typedef enum { LW_SEQ_AUTO = 0, LW_SEQ_PERSISTENT = 1, LW_SEQ_LAUNCHES = 2 } lw_sequence_mode;
+/* Process-wide choice of the implementation behind lw_matvec_sequence; LW_ERR_FORMAT for another value. */
+int lw_set_sequence_mode(int mode);
+
+/* lw_matvec_sequence with HOST activations and results: copies in_bytes from in_host to in_dev (one copy: the
+ * block that holds the chain's input activations; the items' X pointers point into in_dev), runs the chain,
+ * copies out_bytes from out_dev to out_host (the block the items' Y pointers point into), all asynchronously
+ * on `stream` (pinned host memory makes the copies truly asynchronous).  in_dev / out_dev are caller-provided
+ * device buffers; a size of 0 skips that copy.  The caller synchronises the stream before reading out_host.
+ * Errors as lw_matvec_sequence; a call that fails validation enqueues nothing. */
+int lw_matvec_sequence_host(int fmt, int n_items, const lw_seq_item* items, const void* in_host, void* in_dev,
+                            int64_t in_bytes, const void* out_dev, void* out_host, int64_t out_bytes, void* workspace,
+                            int64_t workspace_bytes, void* stream);
 
 /* Kernel-variant selection [Sec 3.2: the kernel library picks a variant from the tensor context;
  * tunable work-group and tile sizes].  LW_VARIANT_AUTO lets the launch heuristics decide. */
@@ -292,6 +309,12 @@ int lw_attn_decode_static(int kv_fmt, const void* K_blocks, const void* V_blocks
  * never trap or spin forever: a bounded wait that gives up records a code here and the kernel
  * finishes.  This call synchronises the device.  Returns LW_OK, LW_ERR_NULL or LW_ERR_CUDA. */
 int lw_device_status(int* status_out);
+
+/* Measurement aid (the paper has no counterpart): streams `bytes` bytes at `src` (device, 16-byte aligned, a
+ * multiple of 16 bytes) through the copy pipeline of the streaming mat-vec kernels -- one CTA per SM, rings of
+ * 1-D bulk copies into shared memory, L2 evict-first -- and does nothing with them.  Timing it gives the
+ * read-only bandwidth ceiling of that pipeline on the device.  Asynchronous on `stream`. */
+int lw_probe_read(const void* src, int64_t bytes, void* stream);
 
 /* Testing aid for that fault path (the paper has no counterpart).  After lw_debug_drop_copy(u), u >= 0, the
  * next batch-1 lw_matvec that takes a streaming kernel never requests the copy of the u-th row unit of each

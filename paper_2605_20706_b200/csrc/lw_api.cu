@@ -10,6 +10,7 @@ namespace lw {
 
 static std::atomic<int> g_variant{-1};   // -1: not initialised (environment not read yet)
 static std::atomic<int> g_overlap{0};
+static std::atomic<int> g_sequence_mode{LW_SEQ_AUTO};
 
 static int forced_variant() {
     int v = g_variant.load(std::memory_order_relaxed);
@@ -229,15 +230,75 @@ int lw_matvec_sequence(int fmt, int n_items, const lw_seq_item* items, void* wor
         coop[dev] = (cudaDeviceGetAttribute(&v, cudaDevAttrCooperativeLaunch, dev) == cudaSuccess && v) ? 1 : -1;
     }
     const bool can = dev >= 0 && dev < 64 && coop[dev] == 1;
-    if (can && forced_variant() == LW_VARIANT_AUTO && matvec_sequence_supported(fmt, n_items, items)) {
-        const int err = launch_matvec_sequence(fmt, n_items, items, static_cast<unsigned*>(workspace),
-                                               static_cast<cudaStream_t>(stream));
+    const bool streaming = forced_variant() == LW_VARIANT_AUTO && matvec_sequence_supported(fmt, n_items, items);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (streaming && can && g_sequence_mode.load() == LW_SEQ_PERSISTENT) {
+        const int err = launch_matvec_sequence(fmt, n_items, items, static_cast<unsigned*>(workspace), s);
         return err == 0 ? LW_OK : LW_ERR_CUDA;
+    }
+    if (streaming) {
+        // One launch per phase (consecutive items that share their X and are not flagged dependent), chained
+        // with programmatic dependent launch: stream order provides every dependency, and a kernel waits for
+        // its predecessor before it requests any of W or X.
+        int j = 0;
+        while (j < n_items) {
+            int n = 1;
+            while (j + n < n_items && n < 8 && !(items[j + n].flags & LW_SEQ_DEPENDENT) && items[j + n].X == items[j].X &&
+                   items[j + n].cols == items[j].cols)
+                ++n;
+            const void* W[8];
+            const float* X[8];
+            float* Y[8];
+            int64_t rows[8];
+            for (int k = 0; k < n; ++k) {
+                W[k] = items[j + k].W_blocks;
+                X[k] = items[j + k].X;
+                Y[k] = items[j + k].Y;
+                rows[k] = items[j + k].rows;
+            }
+            const int err = n == 1 ? launch_matvec_stream(fmt, fmt != LW_F16, W[0], rows[0], items[j].cols, X[0], Y[0], true, s)
+                                   : launch_matvec_stream_group(fmt, fmt != LW_F16, items[j].cols, n, W, rows, X, Y, true, s);
+            if (err != 0) return LW_ERR_CUDA;
+            j += n;
+        }
+        return LW_OK;
     }
     for (int j = 0; j < n_items; ++j) {
         const int rc = lw_matvec(fmt, items[j].W_blocks, items[j].rows, items[j].cols, items[j].X, items[j].Y, 1, stream);
         if (rc != LW_OK) return rc;
     }
+    return LW_OK;
+}
+
+int lw_matvec_sequence_host(int fmt, int n_items, const lw_seq_item* items, const void* in_host, void* in_dev,
+                            int64_t in_bytes, const void* out_dev, void* out_host, int64_t out_bytes, void* workspace,
+                            int64_t workspace_bytes, void* stream) {
+    if (!in_host || !in_dev || !out_dev || !out_host) return LW_ERR_NULL;
+    if (in_bytes < 0 || out_bytes < 0) return LW_ERR_SHAPE;
+    // validate everything before the first copy is queued: a call that fails enqueues nothing
+    if (lw_block_elems(fmt) == 0) return LW_ERR_FORMAT;
+    if (!items || !workspace) return LW_ERR_NULL;
+    if (n_items < 1 || n_items > 640) return LW_ERR_SHAPE;
+    if (misaligned16(workspace)) return LW_ERR_ALIGN;
+    if (workspace_bytes < lw_matvec_sequence_workspace_bytes()) return LW_ERR_WORKSPACE;
+    for (int j = 0; j < n_items; ++j) {
+        const int rc = check_matvec_args(fmt, items[j].W_blocks, items[j].rows, items[j].cols, items[j].X, items[j].Y, 1);
+        if (rc != LW_OK) return rc;
+        if (items[j].flags & ~LW_SEQ_DEPENDENT) return LW_ERR_FORMAT;
+    }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (in_bytes > 0 && cudaMemcpyAsync(in_dev, in_host, (size_t)in_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess)
+        return LW_ERR_CUDA;
+    const int rc = lw_matvec_sequence(fmt, n_items, items, workspace, workspace_bytes, stream);
+    if (rc != LW_OK) return rc;
+    if (out_bytes > 0 && cudaMemcpyAsync(out_host, out_dev, (size_t)out_bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess)
+        return LW_ERR_CUDA;
+    return LW_OK;
+}
+
+int lw_set_sequence_mode(int mode) {
+    if (mode < LW_SEQ_AUTO || mode > LW_SEQ_LAUNCHES) return LW_ERR_FORMAT;
+    g_sequence_mode.store(mode);
     return LW_OK;
 }
 
@@ -284,6 +345,13 @@ int lw_plan_info(int fmt, int64_t rows, int64_t cols, int* out6) {
         for (int i = 0; i < 6; ++i) out6[i] = 0;       // shape not covered by the streaming kernels
     }
     return LW_OK;
+}
+
+int lw_probe_read(const void* src, int64_t bytes, void* stream) {
+    if (!src) return LW_ERR_NULL;
+    if (bytes < 16 || bytes % 16 != 0) return LW_ERR_SHAPE;
+    if (misaligned16(src)) return LW_ERR_ALIGN;
+    return launch_probe_read(src, bytes, static_cast<cudaStream_t>(stream)) == 0 ? LW_OK : LW_ERR_CUDA;
 }
 
 int lw_debug_drop_copy(int unit) {

@@ -41,6 +41,8 @@ int launch_matvec_stream_group(int fmt, bool integer_dot, int64_t cols, int n_it
 // `counter` is a device word owned by the caller (cleared on the stream by the launch).
 bool matvec_sequence_supported(int fmt, int n_items, const lw_seq_item* items);
 int launch_matvec_sequence(int fmt, int n_items, const lw_seq_item* items, unsigned* counter, cudaStream_t stream);
+// Read-only streaming probe over `bytes` bytes (a multiple of 16) at `src`.
+int launch_probe_read(const void* src, int64_t bytes, cudaStream_t stream);
 // Tunables of the streaming kernels (0 = automatic) and the geometry they lead to for a shape.
 void set_stream_tuning(int worker_groups, int stages, int stage_kb);
 // Testing aid: the next single-matrix streaming launch never requests the copy of pool unit `unit` (< 0: none).

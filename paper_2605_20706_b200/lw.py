@@ -31,7 +31,7 @@ EXPORTS = ("lw_block_elems", "lw_block_bytes", "lw_row_bytes", "lw_status_string
            "lw_dequant", "lw_matvec", "lw_matvec_group", "lw_matvec_host", "lw_set_variant", "lw_query_variant",
            "lw_set_overlap", "lw_device_status", "lw_set_tuning", "lw_plan_info", "lw_attn_decode",
            "lw_attn_workspace_bytes", "lw_attn_decode_static", "lw_set_attn_variant", "lw_query_attn_variant",
-           "lw_debug_drop_copy", "lw_matvec_sequence", "lw_matvec_sequence_workspace_bytes")
+           "lw_debug_drop_copy", "lw_matvec_sequence", "lw_matvec_sequence_workspace_bytes", "lw_probe_read", "lw_set_sequence_mode", "lw_matvec_sequence_host")
 
 _lib = None
 
@@ -77,6 +77,10 @@ def lib() -> ctypes.CDLL:
     L.lw_matvec_sequence_workspace_bytes.restype, L.lw_matvec_sequence_workspace_bytes.argtypes = i64, []
     L.lw_matvec_sequence.restype = c_int
     L.lw_matvec_sequence.argtypes = [c_int, c_int, vp, vp, i64, vp]
+    L.lw_set_sequence_mode.restype, L.lw_set_sequence_mode.argtypes = c_int, [c_int]
+    L.lw_matvec_sequence_host.restype = c_int
+    L.lw_matvec_sequence_host.argtypes = [c_int, c_int, vp, vp, vp, i64, vp, vp, i64, vp, i64, vp]
+    L.lw_probe_read.restype, L.lw_probe_read.argtypes = c_int, [vp, i64, vp]
     L.lw_debug_drop_copy.restype, L.lw_debug_drop_copy.argtypes = c_int, [c_int]
     L.lw_attn_decode_static.restype = c_int
     L.lw_attn_decode_static.argtypes = [c_int, vp, vp, vp, vp, i64, i64, i64, i64, ctypes.c_float, vp]
@@ -191,6 +195,24 @@ def matvec_sequence(fmt: int, items, workspace, workspace_bytes: int | None = No
                                     workspace_bytes, _stream_handle(stream)), "lw_matvec_sequence")
 
 
+SEQ_AUTO, SEQ_PERSISTENT, SEQ_LAUNCHES = 0, 1, 2
+
+
+def set_sequence_mode(mode: int) -> None:
+    _check(lib().lw_set_sequence_mode(mode), "lw_set_sequence_mode")
+
+
+def matvec_sequence_host(fmt: int, items, in_host, in_dev, in_bytes: int, out_dev, out_host, out_bytes: int, workspace,
+                         workspace_bytes: int | None = None, stream=None) -> None:
+    """matvec_sequence between one copy of the input block host -> device and one of the output block back."""
+    arr = items if isinstance(items, ctypes.Array) else seq_items(items)
+    if workspace_bytes is None:
+        workspace_bytes = workspace.numel() * workspace.element_size() if hasattr(workspace, "numel") else 0
+    _check(lib().lw_matvec_sequence_host(fmt, len(arr), ctypes.cast(arr, ctypes.c_void_p), _addr(in_host), _addr(in_dev),
+                                         in_bytes, _addr(out_dev), _addr(out_host), out_bytes, _addr(workspace),
+                                         workspace_bytes, _stream_handle(stream)), "lw_matvec_sequence_host")
+
+
 def matvec_host(fmt: int, W_blocks, rows: int, cols: int, X_host, Y_host, X_dev, Y_dev,
                 batch: int = 1, stream=None) -> None:
     _check(lib().lw_matvec_host(fmt, _addr(W_blocks), rows, cols, _addr(X_host), _addr(Y_host),
@@ -259,6 +281,11 @@ def plan_info(fmt: int, rows: int, cols: int) -> dict:
     _check(lib().lw_plan_info(fmt, rows, cols, ctypes.cast(out, ctypes.c_void_p)), "lw_plan_info")
     keys = ("worker_groups", "stages", "stage_rows", "stage_bytes", "ctas", "smem_bytes")
     return dict(zip(keys, list(out)))
+
+
+def probe_read(src, nbytes: int, stream=None) -> None:
+    """Measurement aid: streams nbytes at src through the streaming kernels' copy pipeline, no arithmetic."""
+    _check(lib().lw_probe_read(_addr(src), nbytes, _stream_handle(stream)), "lw_probe_read")
 
 
 def debug_drop_copy(unit: int) -> None:

@@ -13,6 +13,16 @@ from gpu_util import Guarded, check_matvec, quantized_weights
 torch = pytest.importorskip("torch")
 pytestmark = pytest.mark.gpu
 
+MODES = [lw.SEQ_PERSISTENT, lw.SEQ_LAUNCHES]
+
+
+@pytest.fixture(autouse=True)
+def _reset_mode():
+    yield
+    lw.set_sequence_mode(lw.SEQ_AUTO)
+    lw.set_variant(lw.VARIANT_AUTO)
+
+
 FMTS = [lw.F16, lw.Q8_0, lw.Q4_0, lw.Q4_K, lw.Q6_K, lw.Q5_K, lw.Q2_K, lw.Q4_1, lw.Q5_0, lw.Q5_1]
 DEP = lw.SEQ_DEPENDENT
 
@@ -45,9 +55,11 @@ def _layer_like(fmt, cols_a, cols_b, seed, scale_rows=1):
     return items, keep, refs
 
 
+@pytest.mark.parametrize("mode", MODES)
 @pytest.mark.parametrize("fmt", FMTS)
 @pytest.mark.parametrize("cols_a,cols_b", [(4096, 14336), (2048, 8192), (256, 512)])
-def test_sequence_of_layer_shaped_items(fmt, cols_a, cols_b):
+def test_sequence_of_layer_shaped_items(fmt, cols_a, cols_b, mode):
+    lw.set_sequence_mode(mode)
     if fmt == lw.Q6_K and (cols_a % 2048 or cols_b % 2048):
         cols_a, cols_b = 2048, 6144          # q6_K rows must be whole 16-byte pieces for the streaming kernels
     if fmt == lw.Q2_K and (cols_a % 1024 or cols_b % 1024):
@@ -64,8 +76,10 @@ def test_sequence_of_layer_shaped_items(fmt, cols_a, cols_b):
         check_matvec(y.t.cpu().numpy(), y_ref, s_ref, "sequence item")
 
 
+@pytest.mark.parametrize("mode", MODES)
 @pytest.mark.parametrize("fmt", [lw.Q4_K, lw.Q8_0, lw.F16, lw.Q4_0, lw.Q6_K])
-def test_chain_where_every_item_reads_the_previous_result(fmt):
+def test_chain_where_every_item_reads_the_previous_result(fmt, mode):
+    lw.set_sequence_mode(mode)
     # item i+1's X is item i's Y: the grid-wide barrier before a dependent item is what makes this right.
     # Each stage is checked against the oracle applied to the GPU's own previous stage (fp32), so errors
     # do not compound in the comparison.
@@ -102,6 +116,47 @@ def test_chain_where_every_item_reads_the_previous_result(fmt):
         y_ref, s_ref = oracle.matvec(fmt, blocks, rows, cols, x_prev, 1, nthreads=8)
         check_matvec(got, y_ref, s_ref, "chain stage %d" % i)
         x_prev = got.astype(np.float32)
+
+
+@pytest.mark.parametrize("mode", MODES)
+def test_sequence_with_host_buffers(mode):
+    # lw_matvec_sequence_host: the input block comes from pinned host memory in one copy, the result block
+    # goes back in one copy; the items point into the device blocks
+    lw.set_sequence_mode(mode)
+    fmt = lw.Q4_K
+    spec = [(300, 4096, 0, 0), (77, 4096, 0, 0), (512, 4096, 1, DEP), (129, 2048, 2, DEP)]     # rows, cols, which x, flags
+    xs = [synth.activations(150, i, 1, c) for i, c in ((0, 4096), (1, 4096), (2, 2048))]
+    xoff = [0, 4096, 8192]
+    in_host = torch.from_numpy(np.concatenate([x.reshape(-1) for x in xs])).pin_memory()
+    in_dev = Guarded(in_host.numel())
+    yoff, total = [], 0
+    for rows, _, _, _ in spec:
+        yoff.append(total)
+        total += (rows + 63) & ~63
+    out_dev = Guarded(total)
+    out_host = torch.full((total,), float("nan"), dtype=torch.float32).pin_memory()
+    items, refs, keep = [], [], []
+    for j, (rows, cols, xi, flags) in enumerate(spec):
+        blocks = quantized_weights(fmt, rows, cols, seed=151 + j)
+        w = torch.from_numpy(blocks).cuda()
+        keep.append(w)
+        items.append((w, rows, cols, in_dev.t.data_ptr() + 4 * xoff[xi], out_dev.t.data_ptr() + 4 * yoff[j], flags))
+        refs.append(oracle.matvec(fmt, blocks, rows, cols, xs[xi], 1, nthreads=4))
+    ws = _workspace()
+    for _ in range(2):
+        lw.matvec_sequence_host(fmt, items, in_host, in_dev.t, 4 * in_host.numel(), out_dev.t, out_host, 4 * total, ws.t)
+    torch.cuda.synchronize()
+    assert lw.device_status() == 0
+    in_dev.check("device input block")
+    out_dev.check("device output block")
+    for j, (rows, _, _, _) in enumerate(spec):
+        check_matvec(out_host.numpy()[yoff[j]:yoff[j] + rows], refs[j][0], refs[j][1], "host sequence item %d" % j)
+    L = lw.lib()
+    import ctypes
+    arr = lw.seq_items(items)
+    assert L.lw_matvec_sequence_host(fmt, len(items), ctypes.cast(arr, ctypes.c_void_p), None, in_dev.t.data_ptr(), 16,
+                                     out_dev.t.data_ptr(), out_host.data_ptr(), 16, ws.t.data_ptr(), 256, None) == lw.ERR_NULL
+    assert L.lw_set_sequence_mode(7) == lw.ERR_FORMAT
 
 
 def test_sequence_falls_back_for_shapes_outside_the_streaming_kernels():
