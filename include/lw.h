@@ -211,19 +211,26 @@ typedef enum {
                                512-thread CTA per SM; needs cols % 256 == 0, cols <= 16384 and rows that are
                                whole 16-byte pieces; batch 1.  Exists for f16, q8_0, q4_0 and q4_K; forced on
                                one of the six later formats it falls back to LW_VARIANT_GENERIC */
-    LW_VARIANT_IDOT = 3     /* same streaming skeleton, but activations are converted once per call to
+    LW_VARIANT_IDOT = 3,    /* same streaming skeleton, but activations are converted once per call to
                                24-bit block fixed point (one fp32 scale per 16 or 32 values) and the
                                products run as exact integer dot products (dp4a); error per
                                activation <= 2^-22 of its group's largest magnitude (see the accuracy
                                statement of lw_matvec).  All nine quantised formats (f16 falls back to
                                LW_VARIANT_STREAM).  q8_0, q4_0 and q4_K also have a batched form (2..16
                                columns, fixed-point activations kept in shared memory) */
+    LW_VARIANT_TILE = 4     /* batch 2..16 only: fp32 tile kernel, a lane owns rows, every weight is decoded once
+                               (exactly) and multiplied with all columns of a pass (up to 8) by packed fp32 FMAs,
+                               activations read from shared memory by broadcast; q8_0 and q4_0, cols a multiple
+                               of 1024.  E = 0 in the accuracy statement of lw_matvec; a row's sum is completed
+                               with atomic additions (one per 1024 columns), so the last bits of a result can
+                               differ from run to run.  AUTO takes it from 7 columns on (passes of 7 or 8 columns;
+                               a remainder of fewer goes through the batch-1 kernel column by column) */
 } lw_variant;
 /* Process-wide; returns LW_ERR_FORMAT for an unknown value.  Also settable once at load time
  * through the environment variable LW_FORCE_VARIANT (a number).  A forced variant that does not
  * support the problem (shape, batch, format) falls back to the next simpler one.  AUTO picks, when
- * the shape qualifies: IDOT for the quantised formats (batch 2..16: its batch-1 kernel once per
- * column), STREAM for f16 up to batch 4 (likewise); otherwise GENERIC. */
+ * the shape qualifies: IDOT for the quantised formats (batch 2..16: TILE from 7 columns on where it applies,
+ * else IDOT's batch-1 kernel once per column), STREAM for f16 up to batch 4 (likewise); otherwise GENERIC. */
 int lw_set_variant(int variant);
 /* The variant lw_matvec would launch for this problem (after forcing and shape checks), or a
  * negative lw_status. */

@@ -43,6 +43,11 @@ bool matvec_sequence_supported(int fmt, int n_items, const lw_seq_item* items);
 int launch_matvec_sequence(int fmt, int n_items, const lw_seq_item* items, unsigned* counter, cudaStream_t stream);
 // Read-only streaming probe over `bytes` bytes (a multiple of 16) at `src`.
 int launch_probe_read(const void* src, int64_t bytes, cudaStream_t stream);
+// Batched fp32 tile kernel (2..16 columns, every decoded weight used for all columns of a pass): q8_0 and
+// q4_0, cols a multiple of 1024.
+bool matvec_tile_supported(int fmt, int64_t rows, int64_t cols, int batch);
+int launch_matvec_tile(int fmt, const void* W, int64_t rows, int64_t cols, const float* X, float* Y, int batch,
+                       cudaStream_t stream);
 // Tunables of the streaming kernels (0 = automatic) and the geometry they lead to for a shape.
 void set_stream_tuning(int worker_groups, int stages, int stage_kb);
 // Testing aid: the next single-matrix streaming launch never requests the copy of pool unit `unit` (< 0: none).

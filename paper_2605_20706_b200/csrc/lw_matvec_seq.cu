@@ -161,7 +161,7 @@ __device__ __forceinline__ void walker_take(const SeqParams& p, Walker& w, int w
 // must not weigh on the allocation of the product loop.
 template <int GROUP, bool Q4K_LAYOUT>
 __device__ __noinline__ void seq_convert_activations(const float* X, int cols, uint32_t* xq, int tid) {
-    quantize_activations8<GROUP, Q4K_LAYOUT, 2 * kThreads>(X, cols, xq, tid);
+    quantize_activations8<GROUP, Q4K_LAYOUT, 2 * kThreads, true>(X, cols, xq, tid, [] {});
 }
 
 // One claim of a producer thread: the group's next unit (n == 0 when its list is exhausted).

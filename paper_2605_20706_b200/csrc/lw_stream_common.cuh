@@ -375,10 +375,12 @@ __device__ __forceinline__ void quantize_activations(const float* __restrict__ X
 // The same conversion with 8 values per thread (two lanes share a run of 16, four a group of 32): half the
 // loads and arithmetic per thread and twice the threads at work for vectors of up to 8 * NTHREADS columns,
 // which is what matters when the conversion sits on the critical path between two dependent mat-vecs.
-// Always reads X past the L1 cache (it may have been written by other SMs earlier in the same launch).
+// COHERENT reads X past the L1 cache (it may have been written by other SMs earlier in the same launch).
+// `after_first_loads()` is called once per thread that has a piece, right after its first loads are issued.
 // cols is a multiple of 256, NTHREADS a multiple of 32: whole warps take part or drop out together.
-template <int GROUP, bool Q4K_LAYOUT, int NTHREADS>
-__device__ __forceinline__ void quantize_activations8(const float* __restrict__ X, int cols, uint32_t* xq, int tid) {
+template <int GROUP, bool Q4K_LAYOUT, int NTHREADS, bool COHERENT = true, class AfterLoads>
+__device__ __forceinline__ void quantize_activations8(const float* __restrict__ X, int cols, uint32_t* xq, int tid,
+                                                      AfterLoads after_first_loads) {
     const int pieces = cols >> 3;
     constexpr int kDepth = 2;            // pieces whose loads are in flight together
     for (int p0 = tid; p0 < pieces; p0 += kDepth * NTHREADS) {
@@ -387,10 +389,12 @@ __device__ __forceinline__ void quantize_activations8(const float* __restrict__ 
         for (int j = 0; j < kDepth; ++j) {
             const int piece = p0 + j * NTHREADS;
             if (piece < pieces) {
-                lo[j] = __ldcg(reinterpret_cast<const float4*>(X) + 2 * piece);
-                hi[j] = __ldcg(reinterpret_cast<const float4*>(X) + 2 * piece + 1);
+                const float4* src = reinterpret_cast<const float4*>(X) + 2 * piece;
+                lo[j] = COHERENT ? __ldcg(src) : __ldg(src);
+                hi[j] = COHERENT ? __ldcg(src + 1) : __ldg(src + 1);
             }
         }
+        if (p0 == tid) after_first_loads();
 #pragma unroll
         for (int j = 0; j < kDepth; ++j) {
             const int piece = p0 + j * NTHREADS;

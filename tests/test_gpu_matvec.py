@@ -62,6 +62,27 @@ def test_matvec_batched(variant, fmt, batch):
     check_matvec(y, y_ref, s_ref, "fmt %d batch %d" % (fmt, batch))
 
 
+@pytest.mark.parametrize("fmt", [lw.Q8_0, lw.Q4_0])
+@pytest.mark.parametrize("batch", [2, 3, 4, 5, 8, 9, 13, 16])
+@pytest.mark.parametrize("rows,cols", [(1, 1024), (63, 2048), (64, 1024), (65, 4096), (333, 3072), (1000, 14336),
+                                       (70000, 1024)])
+def test_matvec_tile_kernel(fmt, batch, rows, cols):
+    # the batched fp32 tile kernel (AUTO's choice for q8_0 / q4_0 when cols is a multiple of 1024): ragged row
+    # counts around its 64-row stages, one to fourteen column chunks, passes of 4 and 8 columns, several CTAs
+    # per SM (70000 rows); forced and automatic selection must agree
+    lw.set_variant(lw.VARIANT_AUTO)
+    assert lw.query_variant(fmt, rows, cols, batch) == (lw.VARIANT_TILE if batch >= 7 else lw.VARIANT_IDOT)
+    lw.set_variant(lw.VARIANT_TILE)
+    assert lw.query_variant(fmt, rows, cols, batch) == lw.VARIANT_TILE
+    blocks = quantized_weights(fmt, rows, cols, seed=59, tensor_id=fmt, outlier_p=0.01)
+    X = synth.activations(59, batch, batch, cols)
+    y_ref, s_ref = oracle.matvec(fmt, blocks, rows, cols, X, batch, nthreads=8)
+    y = gpu_matvec(fmt, blocks, rows, cols, X, batch, lw.VARIANT_TILE)
+    check_matvec(y, y_ref, s_ref, "tile fmt %d %dx%d batch %d" % (fmt, rows, cols, batch))
+    y = gpu_matvec(fmt, blocks, rows, cols, X, batch, lw.VARIANT_AUTO)      # tile passes + a column-wise remainder
+    check_matvec(y, y_ref, s_ref, "auto fmt %d %dx%d batch %d" % (fmt, rows, cols, batch))
+
+
 @pytest.mark.parametrize("variant", VARIANTS)
 def test_config1_q8_0_2048(variant):
     # the single q8_0 mat-vec of the first benchmark configuration: every output checked
