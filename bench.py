@@ -301,6 +301,8 @@ def run_step(args):
     Y = torch.zeros(yt, dtype=torch.float32, device="cuda")
 
     lw.set_overlap(not args.no_overlap)
+    if args.tuning_table:
+        log("tuning table: %d entries" % lw.load_tuning_table(args.tuning_table))
     wptr, xptr, yptr = W.data_ptr(), X.data_ptr(), Y.data_ptr()
     xhptr, yhptr = X_host.data_ptr(), Y_host.data_ptr()
 
@@ -1158,6 +1160,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=4.0)
     ap.add_argument("--ref-rows", type=int, default=512)
+    ap.add_argument("--tuning-table", default=None, help="per-shape table written by the autotune sweep, installed before the run")
     args = ap.parse_args()
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ and args.impl == "ours":
         spawn_ranks(args)

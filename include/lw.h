@@ -244,6 +244,15 @@ int lw_query_variant(int fmt, int64_t rows, int64_t cols, int batch);
  * the environment variables LW_WORKER_GROUPS, LW_STAGES, LW_STAGE_KB give the initial values.
  * Returns LW_ERR_FORMAT for values outside 0..2, 0..4, 0..96. */
 int lw_set_tuning(int worker_groups, int stages, int stage_kb);
+/* The same tunables for ONE shape [Sec 3.2: the kernel library selects a tuned variant from the tensor context;
+ * Sec 3.1: the tuning table comes from an empirical sweep].  The launch heuristics consult these entries for
+ * every parameter that lw_set_tuning leaves at 0; a grouped launch or a sequence phase is looked up by the sum
+ * of its rows.  The sweep (python -m paper_2605_20706_b200.autotune --table FILE) writes the table,
+ * lw.load_tuning_table(FILE) of the Python binding installs it.  All three values 0 removes the entry;
+ * lw_clear_shape_tuning removes all.  Process-wide, meant to be changed between launches. */
+int lw_set_shape_tuning(int fmt, int64_t rows, int64_t cols, int worker_groups, int stages, int stage_kb);
+int lw_clear_shape_tuning(void);
+
 /* What the launch heuristics choose for one batch-1 mat-vec under the current tuning: out6 =
  * {worker groups, ring slots per group, rows per slot, bytes per slot, CTAs, shared memory per CTA};
  * all zero when the shape goes to the generic kernels.  Host only, no CUDA work besides a device

@@ -2,9 +2,12 @@
 models: worker groups per CTA, ring slots per group and ring-slot size (`lw_set_tuning`), timed per
 (format, rows, cols) as back-to-back launches inside a CUDA graph with programmatic dependent launch.
 Writes a Markdown table: per shape the time under the launch heuristics' own choice, the best
-setting found and the ratio between the two.
+setting found, the ratio between the two, and the time of the other kernel family (fp32 activations
+instead of the integer-dot form) where a format has both.  With --table it also writes the per-shape
+table (JSON) of the settings that beat the heuristics by more than 2 %, which `lw.load_tuning_table`
+installs (`lw_set_shape_tuning`) and the launch heuristics then consult.
 
-    python -m paper_2605_20706_b200.autotune --out profiles/autotune_stream_kernels.md
+    python -m paper_2605_20706_b200.autotune --out profiles/autotune_stream_kernels.md --table tuning_table.json
 
 The matrices are seeded synthetic weights quantised with the library's host quantiser (a 1024-row
 slab tiled to the full height: the timing depends on bytes and shapes only); enough copies of each
@@ -34,6 +37,13 @@ def unique_shapes(models):
             if (rows, cols) not in seen:
                 seen.add((rows, cols))
                 out.append(("%s %s" % (model, leaf), rows, cols))
+        # the grouped launches of a step are planned by the sum of their rows
+        by_leaf = {name.split(".")[-1]: (rows, cols) for name, rows, cols in shapes}
+        for label, leaves in (("q+k+v", ("q", "k", "v")), ("gate+up", ("gate", "up"))):
+            rows, cols = sum(by_leaf[l][0] for l in leaves), by_leaf[leaves[0]][1]
+            if (rows, cols) not in seen:
+                seen.add((rows, cols))
+                out.append(("%s %s" % (model, label), rows, cols))
     return out
 
 
@@ -72,6 +82,7 @@ def main():
     ap.add_argument("--formats", default="q4_K,q4_0,q8_0,f16")
     ap.add_argument("--models", default="8b,1b")
     ap.add_argument("--out", default=None)
+    ap.add_argument("--table", default=None, help="write the per-shape table of winning settings (JSON) here")
     ap.add_argument("--launches", type=int, default=24)
     ap.add_argument("--replays", type=int, default=6)
     args = ap.parse_args()
@@ -81,8 +92,8 @@ def main():
         raise SystemExit("autotune needs a CUDA device")
     lw.set_overlap(True)
     lines = ["| format | matrix | rows x cols | heuristics: groups/slots/slot KB | us | best: groups/slots/slot KB | us | "
-             "heuristics / best |", "|---|---|---|---|---|---|---|---|"]
-    grids = []
+             "heuristics / best | fp32-activation family us |", "|---|---|---|---|---|---|---|---|---|"]
+    grids, table = [], []
     for fname in args.formats.split(","):
         fmt = lw.FORMATS[fname]
         for label, rows, cols in unique_shapes(args.models.split(",")):
@@ -104,11 +115,21 @@ def main():
                     continue                       # not feasible, or the same geometry as an earlier setting
                 results[key] = (time_setting(torch, fmt, rows, cols, ws, x, ys, launches, args.replays), (g, s, kb))
             lw.set_tuning()
+            other = None
+            if fname in ("q8_0", "q4_0", "q4_K"):              # the variant is a tunable too: the fp32-activation family
+                lw.set_variant(lw.VARIANT_STREAM)
+                other = time_setting(torch, fmt, rows, cols, ws, x, ys, launches, args.replays)
+                lw.set_variant(lw.VARIANT_AUTO)
             best_key = min(results, key=lambda k: results[k][0])
             best_us = results[best_key][0]
-            lines.append("| %s | %s | %d x %d | %d/%d/%.0f | %.2f | %d/%d/%.0f | %.2f | %.3f |" % (
+            if base / best_us > 1.02:
+                g, s, kb = results[best_key][1]
+                table.append({"format": fname, "rows": rows, "cols": cols, "worker_groups": g, "stages": s, "stage_kb": kb,
+                              "us_heuristics": round(base, 2), "us_tuned": round(best_us, 2)})
+            lines.append("| %s | %s | %d x %d | %d/%d/%.0f | %.2f | %d/%d/%.0f | %.2f | %.3f | %s |" % (
                 fname, label, rows, cols, info["worker_groups"], info["stages"], info["stage_bytes"] / 1024, base,
-                best_key[0], best_key[1], best_key[2] / 1024, best_us, base / best_us))
+                best_key[0], best_key[1], best_key[2] / 1024, best_us, base / best_us,
+                "%.2f" % other if other is not None else "-"))
             grids.append((fname, label, rows, cols, results))
             print(lines[-1], file=sys.stderr, flush=True)
             del ws
@@ -126,6 +147,10 @@ def main():
         text.append("%s, %s (%d x %d): groups/slots/slot KB -> us: " % (fname, label, rows, cols) + ", ".join(
             "%d/%d/%.0f %.2f" % (k[0], k[1], k[2] / 1024, v[0]) for k, v in sorted(results.items(), key=lambda kv: kv[1][0])))
         text.append("")
+    if args.table:
+        import json
+        with open(args.table, "w") as fh:
+            json.dump(table, fh, indent=1)
     out = "\n".join(text)
     if args.out:
         with open(args.out, "w") as fh:

@@ -356,6 +356,20 @@ int lw_set_tuning(int worker_groups, int stages, int stage_kb) {
     return LW_OK;
 }
 
+int lw_set_shape_tuning(int fmt, int64_t rows, int64_t cols, int worker_groups, int stages, int stage_kb) {
+    if (lw_block_elems(fmt) == 0) return LW_ERR_FORMAT;
+    if (rows < 1 || lw_row_bytes(fmt, cols) == 0) return LW_ERR_SHAPE;
+    if (worker_groups < 0 || worker_groups > 2 || stages < 0 || stages > 4 || stage_kb < 0 || stage_kb > 96)
+        return LW_ERR_FORMAT;
+    set_shape_tuning(fmt, rows, cols, worker_groups, stages, stage_kb);
+    return LW_OK;
+}
+
+int lw_clear_shape_tuning(void) {
+    clear_shape_tuning();
+    return LW_OK;
+}
+
 int lw_plan_info(int fmt, int64_t rows, int64_t cols, int* out6) {
     if (lw_block_elems(fmt) == 0) return LW_ERR_FORMAT;
     if (!out6) return LW_ERR_NULL;

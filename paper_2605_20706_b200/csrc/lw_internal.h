@@ -50,6 +50,9 @@ int launch_matvec_tile(int fmt, const void* W, int64_t rows, int64_t cols, const
                        cudaStream_t stream);
 // Tunables of the streaming kernels (0 = automatic) and the geometry they lead to for a shape.
 void set_stream_tuning(int worker_groups, int stages, int stage_kb);
+// Per-shape tunables (all zero erases the entry); make_plan uses them where the process-wide ones are 0.
+void set_shape_tuning(int fmt, int64_t rows, int64_t cols, int worker_groups, int stages, int stage_kb);
+void clear_shape_tuning();
 // Testing aid: the next single-matrix streaming launch never requests the copy of pool unit `unit` (< 0: none).
 void set_drop_unit(int unit);
 bool stream_plan_info(int fmt, int64_t rows, int64_t cols, int* groups, int* stages, int* stage_rows, int* stage_bytes,

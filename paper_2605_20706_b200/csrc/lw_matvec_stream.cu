@@ -26,6 +26,7 @@
 #include <atomic>
 #include <cstdlib>
 #include <type_traits>
+#include <vector>
 
 #include "lw_internal.h"
 #include "lw_stream_common.cuh"
@@ -557,6 +558,18 @@ Tuning& tuning_storage() {
 }
 const Tuning& tuning() { return tuning_storage(); }
 
+// Per-shape settings found by a sweep (lw_set_shape_tuning, filled from the table the sweep writes): consulted
+// by make_plan for every parameter the process-wide tuning leaves to the heuristics.
+struct ShapeTuning {
+    int fmt;
+    int64_t rows, cols;
+    int groups, stages, stage_kb;
+};
+std::vector<ShapeTuning>& shape_table() {
+    static std::vector<ShapeTuning> t;
+    return t;
+}
+
 // Testing aid (lw_debug_drop_copy): the next batch-1 streaming launch leaves out the copy of one unit.
 std::atomic<int>& drop_unit_storage() {
     static std::atomic<int> v{-1};
@@ -585,7 +598,13 @@ Plan make_plan(int fmt, bool integer_dot, int64_t rows, int64_t cols, int num_sm
     size_t x_bytes = (size_t)(cols + (xchunk ? 4 * (cols / xchunk) : 0)) * 4u;     // padded fp32 staging
     const bool idot = (integer_dot && fmt != LW_F16) || fmt >= LW_Q6_K;   // the later formats have the integer-dot trait only
     if (idot) x_bytes = ((size_t)units * kXqUnitWords + (kquant ? (size_t)(units / 4) * 4 : 0)) * 4u;
-    const Tuning& tn = tuning();
+    Tuning tn = tuning();
+    for (const ShapeTuning& e : shape_table())
+        if (e.fmt == fmt && e.rows == rows && e.cols == cols) {
+            if (tn.groups == 0) tn.groups = e.groups;
+            if (tn.stages == 0) tn.stages = e.stages;
+            if (tn.stage_kb == 0) tn.stage_kb = e.stage_kb;
+        }
     // One CTA per SM made of two worker groups (512 threads) by default; LW_WORKER_GROUPS=1 selects
     // single-group CTAs instead, two per SM (the decode routines need more than 80 registers to
     // schedule well, so not three), or one per SM with larger stages for rows wider than 8192 columns.
@@ -769,6 +788,18 @@ int batched_columns(int fmt, int64_t rows, int64_t cols) {
 }  // namespace
 
 void set_drop_unit(int unit) { drop_unit_storage().store(unit < 0 ? -1 : unit); }
+
+void set_shape_tuning(int fmt, int64_t rows, int64_t cols, int worker_groups, int stages, int stage_kb) {
+    std::vector<ShapeTuning>& t = shape_table();
+    for (size_t i = 0; i < t.size(); ++i)
+        if (t[i].fmt == fmt && t[i].rows == rows && t[i].cols == cols) {
+            t.erase(t.begin() + (long)i);
+            break;
+        }
+    if (worker_groups != 0 || stages != 0 || stage_kb != 0) t.push_back(ShapeTuning{fmt, rows, cols, worker_groups, stages, stage_kb});
+}
+
+void clear_shape_tuning() { shape_table().clear(); }
 
 void set_stream_tuning(int worker_groups, int stages, int stage_kb) {
     Tuning& t = tuning_storage();

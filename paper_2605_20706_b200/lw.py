@@ -31,7 +31,7 @@ EXPORTS = ("lw_block_elems", "lw_block_bytes", "lw_row_bytes", "lw_status_string
            "lw_dequant", "lw_matvec", "lw_matvec_group", "lw_matvec_host", "lw_set_variant", "lw_query_variant",
            "lw_set_overlap", "lw_device_status", "lw_set_tuning", "lw_plan_info", "lw_attn_decode",
            "lw_attn_workspace_bytes", "lw_attn_decode_static", "lw_set_attn_variant", "lw_query_attn_variant",
-           "lw_debug_drop_copy", "lw_matvec_sequence", "lw_matvec_sequence_workspace_bytes", "lw_probe_read", "lw_set_sequence_mode", "lw_matvec_sequence_host")
+           "lw_debug_drop_copy", "lw_matvec_sequence", "lw_matvec_sequence_workspace_bytes", "lw_probe_read", "lw_set_sequence_mode", "lw_matvec_sequence_host", "lw_set_shape_tuning", "lw_clear_shape_tuning")
 
 _lib = None
 
@@ -68,6 +68,8 @@ def lib() -> ctypes.CDLL:
     L.lw_set_overlap.restype, L.lw_set_overlap.argtypes = c_int, [c_int]
     L.lw_device_status.restype, L.lw_device_status.argtypes = c_int, [vp]
     L.lw_set_tuning.restype, L.lw_set_tuning.argtypes = c_int, [c_int, c_int, c_int]
+    L.lw_set_shape_tuning.restype, L.lw_set_shape_tuning.argtypes = c_int, [c_int, i64, i64, c_int, c_int, c_int]
+    L.lw_clear_shape_tuning.restype, L.lw_clear_shape_tuning.argtypes = c_int, []
     L.lw_plan_info.restype, L.lw_plan_info.argtypes = c_int, [c_int, i64, i64, vp]
     L.lw_attn_workspace_bytes.restype, L.lw_attn_workspace_bytes.argtypes = i64, [i64, i64, i64, i64]
     L.lw_attn_decode.restype = c_int
@@ -274,6 +276,26 @@ def set_overlap(enabled: bool) -> None:
 
 def set_tuning(worker_groups: int = 0, stages: int = 0, stage_kb: int = 0) -> None:
     _check(lib().lw_set_tuning(worker_groups, stages, stage_kb), "lw_set_tuning")
+
+
+def set_shape_tuning(fmt: int, rows: int, cols: int, worker_groups: int = 0, stages: int = 0, stage_kb: int = 0) -> None:
+    _check(lib().lw_set_shape_tuning(fmt, rows, cols, worker_groups, stages, stage_kb), "lw_set_shape_tuning")
+
+
+def clear_shape_tuning() -> None:
+    _check(lib().lw_clear_shape_tuning(), "lw_clear_shape_tuning")
+
+
+def load_tuning_table(path: str) -> int:
+    """Installs the per-shape table a sweep wrote (JSON list of {format, rows, cols, worker_groups, stages,
+    stage_kb}); returns the number of entries."""
+    import json
+    with open(path) as fh:
+        table = json.load(fh)
+    for e in table:
+        set_shape_tuning(FORMATS[e["format"]], e["rows"], e["cols"], e.get("worker_groups", 0), e.get("stages", 0),
+                         e.get("stage_kb", 0))
+    return len(table)
 
 
 def plan_info(fmt: int, rows: int, cols: int) -> dict:

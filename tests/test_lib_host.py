@@ -183,6 +183,39 @@ def test_tuning_controls_and_plan_info():
 
 
 
+def test_per_shape_tuning_table(tmp_path):
+    L = lw.lib()
+    try:
+        lw.set_tuning()
+        lw.clear_shape_tuning()
+        auto = lw.plan_info(lw.Q4_K, 512, 2048)
+        other = lw.plan_info(lw.Q4_K, 4096, 4096)
+        lw.set_shape_tuning(lw.Q4_K, 512, 2048, 1, 2, 45)
+        tuned = lw.plan_info(lw.Q4_K, 512, 2048)
+        assert tuned["worker_groups"] == 1 and tuned != auto
+        assert lw.plan_info(lw.Q4_K, 4096, 4096) == other                   # other shapes keep the heuristics
+        assert lw.plan_info(lw.Q4_0, 512, 2048)["worker_groups"] == 2       # and so do other formats
+        lw.set_tuning(2, 0, 0)                                              # an explicit process-wide value wins
+        assert lw.plan_info(lw.Q4_K, 512, 2048)["worker_groups"] == 2
+        lw.set_tuning()
+        lw.set_shape_tuning(lw.Q4_K, 512, 2048)                             # all zero: entry removed
+        assert lw.plan_info(lw.Q4_K, 512, 2048) == auto
+        # the table file the sweep writes
+        path = tmp_path / "table.json"
+        path.write_text('[{"format": "q8_0", "rows": 512, "cols": 2048, "worker_groups": 1, "stages": 2, "stage_kb": 34, '
+                        '"us_heuristics": 3.0, "us_tuned": 2.8}]')
+        assert lw.load_tuning_table(str(path)) == 1
+        assert lw.plan_info(lw.Q8_0, 512, 2048)["worker_groups"] == 1
+        lw.clear_shape_tuning()
+        assert lw.plan_info(lw.Q8_0, 512, 2048)["worker_groups"] == 2
+        assert L.lw_set_shape_tuning(77, 4, 64, 0, 0, 0) == lw.ERR_FORMAT
+        assert L.lw_set_shape_tuning(lw.Q8_0, 4, 48, 0, 0, 0) == lw.ERR_SHAPE
+        assert L.lw_set_shape_tuning(lw.Q8_0, 4, 64, 3, 0, 0) == lw.ERR_FORMAT
+    finally:
+        lw.set_tuning()
+        lw.clear_shape_tuning()
+
+
 def test_attn_host_side_checks():
     L = lw.lib()
     assert lw.attn_workspace_bytes(32, 8, 128, 8192) == 32 * 256 * 130 * 4
