@@ -1038,7 +1038,9 @@ def run_attn(args):
     result = {
         "metric": ATTN_METRIC, "value": round(gbs, 1), "unit": "GB/s", "n_gpus": world, "steps": args.steps,
         "warmup": max(3, args.warmup), "ms_per_step": round(step_ms, 5), "higher_is_better": True, "scaling": "weak",
-        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "vs_baseline": None, "dtype": "f32 in/out; f16 tensor-core products of exact cache codes with the query and the "
+                                       "probabilities as high + low f16 pairs, fp32 accumulation and softmax"
+        if variant == 2 else "f32 in/out; exact block decode, fp32 FMA", "data": "synthetic",
         "config": {
             "workload": "%s: %d lw_attn_decode calls per step (one per layer, own K and V cache each), %d query heads "
                         "over %d KV heads of %d dims, %d cached positions in %s (%.1f MB per call)%s" % (

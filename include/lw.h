@@ -333,8 +333,8 @@ int lw_device_status(int* status_out);
 int lw_probe_read(const void* src, int64_t bytes, void* stream);
 
 /* Testing aid for that fault path (the paper has no counterpart).  After lw_debug_drop_copy(u), u >= 0, the
- * next batch-1 lw_matvec that takes a streaming kernel never requests the copy of the u-th row unit of each
- * CTA: nothing is in flight for it, the wait for it runs out after its limit (about 0.1 s), the kernel
+ * next batch-1 lw_matvec of a q4_K matrix that takes the streaming kernel (a separate build of it: the kernels
+ * of ordinary calls carry no trace of this aid) never requests the copy of the u-th row unit of each CTA: nothing is in flight for it, the wait for it runs out after its limit (about 0.1 s), the kernel
  * records a fault, requests nothing further and returns; the rows of that unit and of the units after it are
  * left unwritten.  The request is consumed by that one launch; u < 0 cancels it.  Always returns LW_OK. */
 int lw_debug_drop_copy(int unit);

@@ -241,8 +241,21 @@ cudaError_t launch_merge(const float* ws, float* out, int n_head, int parts, int
 // integer codes of the cache are exact in f16; the block scales d are applied in fp32 -- to the score
 // sums per 32-dim block, and to the probabilities (per position and block) before the second product.
 // One CTA per SM takes a contiguous range of positions for all KV heads; a producer warp copies each stage
-// as groups of rows (bulk copies on mbarriers) with padding chosen for bank-conflict-free fragment loads;
+// as groups of rows (bulk copies on mbarriers) with padding chosen so that the K and V fragment loads are
+// free of bank conflicts (host-side simulation, attn_bank_conflicts; the conflicts a profiler still counts,
+// about 15 % of the shared-memory wavefronts at 32768 positions, belong to the other shared-memory traffic);
 // compute warp w serves KV head w mod n_kv_head and the tiles TPW * (w / n_kv_head) ... of the stage.
+//
+// Why mma.sync and not tcgen05.  The M of both products is 8 (four query heads x high | low part) per KV
+// head.  tcgen05.mma needs M = 64 or 128 with A read through a shared-memory descriptor in its canonical
+// (swizzled core-matrix) layout and D in TMEM.  For the code-valued caches (q8_0, q4_0) A would first have to
+// be decoded into that layout -- a second pass over every byte through shared memory, which is what the
+// register decode avoids.  For the f16 cache the scores could take a K tile as A as stored (a tensor-map
+// copy can produce the layout), but the second product has the cached positions as its K dimension and
+// the probabilities as the operand that changes every tile: they would have to go register -> shared memory ->
+// tensor core each tile, with the accumulator read back from TMEM for every rescale, and M padded from 8
+// to 64.  The f16 kernel as it stands is bound by its copies (its time with the arithmetic switched off is
+// within 2 % of the full kernel), so there is nothing for a faster contraction to win there.
 struct AttnMmaParams {
     const uint8_t* K;
     const uint8_t* V;

@@ -90,7 +90,9 @@ struct StreamParams {
 // once per SM, and the two groups finish within one stage of each other whatever share of the issue
 // slots the warp schedulers give them (two independent CTAs on an SM do not: the older one is favoured
 // and the younger one runs its last quarter alone at half the SM's throughput).
-template <class T, int NG>
+// DROP builds the testing aid of lw_debug_drop_copy into the kernel (one copy is never requested); the kernels
+// that serve ordinary calls are built without it, so it costs them nothing.
+template <class T, int NG, bool DROP = false>
 __global__ void __launch_bounds__(NG* kThreads, NG == 1 ? T::kMinCtas : 1)
     matvec_stream_kernel(const StreamParams p) {
     extern __shared__ __align__(128) uint8_t smem[];
@@ -150,7 +152,7 @@ __global__ void __launch_bounds__(NG* kThreads, NG == 1 ? T::kMinCtas : 1)
         mbar_init(xbar, 1);
         *timed_out = 0;
         *unit_counter = 0;
-        *copy_dropped = 0;
+        if constexpr (DROP) *copy_dropped = 0;
         fence_barrier_init();
     }
     __syncthreads();
@@ -166,7 +168,9 @@ __global__ void __launch_bounds__(NG* kThreads, NG == 1 ? T::kMinCtas : 1)
         if constexpr (NG == 1) k = next_unit++;
         else k = atomicAdd(unit_counter, 1);
         int begin = 0, n = 0;
-        if (k < n_units && *copy_dropped == 0) {
+        bool open = true;
+        if constexpr (DROP) open = *copy_dropped == 0;
+        if (k < n_units && open) {
             begin = k < n_short ? k * rows_per_wave : short_rows + (k - n_short) * stage_rows;
             n = rows_here - begin;
             const int cap = k < n_short ? rows_per_wave : stage_rows;
@@ -175,8 +179,11 @@ __global__ void __launch_bounds__(NG* kThreads, NG == 1 ? T::kMinCtas : 1)
         // Testing aid: the copy of one unit is never requested, so the wait for it must run out.  Nothing
         // is queued in the CTA after that (no later copy can land in a slot whose barrier is out of
         // step), and the rows of the units left over are not computed.
-        const bool drop = n > 0 && k == p.drop_unit;
-        if (drop) *copy_dropped = 1;
+        bool drop = false;
+        if constexpr (DROP) {
+            drop = n > 0 && k == p.drop_unit;
+            if (drop) *copy_dropped = 1;
+        }
         {
             uint8_t* rec = smem + rec_base + 16u * (uint32_t)(claims & (kUnitRecords - 1));
             *reinterpret_cast<float**>(rec) = Ym + row0 + begin;
@@ -674,14 +681,14 @@ Plan make_plan(int fmt, bool integer_dot, int64_t rows, int64_t cols, int num_sm
     return pl;
 }
 
-template <class T, int NG>
+template <class T, int NG, bool DROP = false>
 int launch_groups(Plan& pl, bool overlap, cudaStream_t stream) {
     static bool attr_set[64] = {false};
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return (int)e;
     if (dev < 0 || dev >= 64 || !attr_set[dev]) {
-        e = cudaFuncSetAttribute(matvec_stream_kernel<T, NG>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        e = cudaFuncSetAttribute(matvec_stream_kernel<T, NG, DROP>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                  (int)kSmemMaxCta);
         if (e != cudaSuccess) return (int)e;
         if (dev >= 0 && dev < 64) attr_set[dev] = true;
@@ -696,11 +703,14 @@ int launch_groups(Plan& pl, bool overlap, cudaStream_t stream) {
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = overlap ? 1 : 0;
-    return (int)cudaLaunchKernelEx(&cfg, matvec_stream_kernel<T, NG>, pl.p);
+    return (int)cudaLaunchKernelEx(&cfg, matvec_stream_kernel<T, NG, DROP>, pl.p);
 }
 
 template <class T>
 int launch_one(Plan& pl, bool overlap, cudaStream_t stream) {
+    // the testing aid exists in one kernel only (q4_K, two worker groups)
+    if constexpr (std::is_same<T, IdotQ4K>::value)
+        if (pl.p.drop_unit >= 0 && pl.groups == 2) return launch_groups<T, 2, true>(pl, overlap, stream);
     return pl.groups == 2 ? launch_groups<T, 2>(pl, overlap, stream) : launch_groups<T, 1>(pl, overlap, stream);
 }
 

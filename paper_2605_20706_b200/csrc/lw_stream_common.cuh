@@ -325,20 +325,12 @@ __device__ __forceinline__ void quantize_activations(const float* __restrict__ X
             if (run0 + j * NTHREADS >= padded) break;      // warp-uniform: whole warps drop out together
             const int run = run0 + j * NTHREADS;
             const bool valid = run < runs;
-            float amax = 0.f, nonfinite = 0.f;
+            float amax = 0.f;
 #pragma unroll
-            for (int i = 0; i < 16; ++i) {
-                amax = fmaxf(amax, fabsf(v[j][i]));
-                nonfinite = fmaf(v[j][i], 0.f, nonfinite);      // stays 0 unless a value is NaN or Inf
-            }
-            if (GROUP == 32) {
-                amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, 1));
-                nonfinite += __shfl_xor_sync(0xFFFFFFFFu, nonfinite, 1);
-            }
-            // A NaN or Inf activation must reach every output it touches (as in fp32 arithmetic): the
-            // maximum above drops NaNs, so the group's scale is made NaN explicitly.
+            for (int i = 0; i < 16; ++i) amax = fmaxf(amax, fabsf(v[j][i]));
+            if (GROUP == 32) amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, 1));
             const bool nonzero = amax > 1e-30f;
-            const float d = nonfinite != 0.f ? nonfinite : (nonzero ? amax / 4194303.f : 0.f);
+            float d = nonzero ? amax / 4194303.f : 0.f;
             const float inv = nonzero && amax <= 3.0e38f ? 4194303.f / amax : 0.f;
             int q[16];
             int total = 0;
@@ -348,6 +340,14 @@ __device__ __forceinline__ void quantize_activations(const float* __restrict__ X
                 q[i] = __float_as_int(fmaf(v[j][i], inv, 12582912.f)) - 0x4B400000;
                 total += q[i];
             }
+            // A NaN or Inf activation must reach every output it touches (as in fp32 arithmetic), but the
+            // maximum above drops NaNs.  A non-finite value (or a finite one times inv = 0 of an infinite
+            // maximum) leaves a NaN pattern in its code, more than 2^29 away from any sum of 16 proper codes
+            // (|code| <= 2^22), whatever the number of such values: the run's sum gives it away, off the
+            // critical path of the conversion, and the group's scale becomes NaN.
+            int nonfinite = (total > 16 * 4194303 || total < -16 * 4194303) ? 1 : 0;
+            if (GROUP == 32) nonfinite |= __shfl_xor_sync(0xFFFFFFFFu, nonfinite, 1);      // every lane takes part
+            if (nonfinite) d = __int_as_float(0x7FC00000);
             if (valid) {
                 uint32_t* u = xq + xq_unit_offset<Q4K_LAYOUT>(run >> 2);
                 const int jj = run & 3;
@@ -400,22 +400,15 @@ __device__ __forceinline__ void quantize_activations8(const float* __restrict__ 
             const int piece = p0 + j * NTHREADS;
             if (piece >= pieces) break;
             const float v[8] = {lo[j].x, lo[j].y, lo[j].z, lo[j].w, hi[j].x, hi[j].y, hi[j].z, hi[j].w};
-            float amax = 0.f, nonfinite = 0.f;
+            float amax = 0.f;
 #pragma unroll
-            for (int i = 0; i < 8; ++i) {
-                amax = fmaxf(amax, fabsf(v[i]));
-                nonfinite = fmaf(v[i], 0.f, nonfinite);         // stays 0 unless a value is NaN or Inf
-            }
+            for (int i = 0; i < 8; ++i) amax = fmaxf(amax, fabsf(v[i]));
             amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, 1));
-            nonfinite += __shfl_xor_sync(0xFFFFFFFFu, nonfinite, 1);
-            if (GROUP == 32) {
-                amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, 2));
-                nonfinite += __shfl_xor_sync(0xFFFFFFFFu, nonfinite, 2);
-            }
+            if (GROUP == 32) amax = fmaxf(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, 2));
             // scale and its reciprocal without divisions (this sits on a critical path): d * inv may differ from
             // 1 by a few 2^-23, which scales the whole group alike and is far inside the tolerance
             const bool nonzero = amax > 1e-30f;
-            const float d = nonfinite != 0.f ? nonfinite : (nonzero ? amax * (1.f / 4194303.f) : 0.f);
+            float d = nonzero ? amax * (1.f / 4194303.f) : 0.f;
             const float inv = nonzero && amax <= 3.0e38f ? 4194303.f * __frcp_rn(amax) : 0.f;
             int q[8];
             int total = 0;
@@ -424,6 +417,12 @@ __device__ __forceinline__ void quantize_activations8(const float* __restrict__ 
                 q[i] = __float_as_int(fmaf(v[i], inv, 12582912.f)) - 0x4B400000;
                 total += q[i];
             }
+            // non-finite values leave NaN patterns as codes (see quantize_activations): the sum of the thread's
+            // eight codes gives them away; the flag goes to all lanes of the group, whose scale becomes NaN
+            int nonfinite = (total > 8 * 4194303 || total < -8 * 4194303) ? 1 : 0;
+            nonfinite |= __shfl_xor_sync(0xFFFFFFFFu, nonfinite, 1);                       // every lane takes part
+            if (GROUP == 32) nonfinite |= __shfl_xor_sync(0xFFFFFFFFu, nonfinite, 2);
+            if (nonfinite) d = __int_as_float(0x7FC00000);
             total += __shfl_xor_sync(0xFFFFFFFFu, total, 1);      // sum over the run of 16
             const int run = piece >> 1, half = piece & 1;
             uint32_t* u = xq + xq_unit_offset<Q4K_LAYOUT>(run >> 2);

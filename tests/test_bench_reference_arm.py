@@ -12,7 +12,8 @@ KEYS = {"impl", "metric", "value", "unit", "n_gpus", "steps", "warmup", "ms_per_
         "vs_baseline", "dtype", "data", "config", "cpu_baseline", "e2e", "gpu_launches"}
 
 
-@pytest.mark.parametrize("workload,extra", [("llama1b_q4_0", ["--ref-rows", "64"]), ("attn1b_q8_0_ctx8k", [])])
+@pytest.mark.parametrize("workload,extra", [("llama1b_q4_0", ["--ref-rows", "64"]), ("attn1b_q8_0_ctx8k", []),
+                                            ("q8_0_2048", []), ("dequant_q4_K", [])])
 def test_reference_arm_prints_the_contract_line(workload, extra):
     cmd = [sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--workload", workload, "--steps", "1",
            "--warmup", "1"] + extra
@@ -34,3 +35,28 @@ def test_reference_arm_runs_on_rank_zero_only():
                           "attn1b_q8_0_ctx8k", "--steps", "1", "--warmup", "1"], cwd=ROOT, env=env, capture_output=True,
                          text=True, timeout=120, check=True).stdout
     assert out.strip() == ""
+
+
+def test_gpus_flag_without_a_torchrun_environment_starts_the_ranks(monkeypatch):
+    # `python bench.py --gpus N` on its own must not silently run on one GPU: it starts N ranks (torchrun module,
+    # rendezvous on 127.0.0.1) that each run this file with the same arguments
+    import importlib.util
+    spec = importlib.util.spec_from_file_location("bench_module", os.path.join(ROOT, "bench.py"))
+    bench = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(bench)
+    seen = {}
+
+    def fake_call(cmd):
+        seen["cmd"] = cmd
+        return 0
+
+    monkeypatch.setattr(bench.subprocess, "call", fake_call)
+    monkeypatch.setattr(sys, "argv", ["bench.py", "--gpus", "4", "--steps", "7"])
+    monkeypatch.delenv("WORLD_SIZE", raising=False)
+    with pytest.raises(SystemExit) as e:
+        bench.main()
+    assert e.value.code == 0
+    cmd = seen["cmd"]
+    assert cmd[1:3] == ["-m", "torch.distributed.run"]
+    assert cmd[cmd.index("--nproc-per-node") + 1] == "4" and cmd[cmd.index("--master-addr") + 1] == "127.0.0.1"
+    assert cmd[-4:] == ["--gpus", "4", "--steps", "7"] and cmd[-5].endswith("bench.py")

@@ -105,6 +105,14 @@ def test_non_finite_activations_reach_the_output(fmt, variant):
         X[0, where] = bad
         y = _run(fmt, blocks, rows, cols, X, variant)
         assert not np.isfinite(y).any(), "fmt %d variant %d: %r at %d was lost" % (fmt, variant, bad, where)
+    # several non-finite values in one run of 16 (the kernels spot them through a sum of integer codes that wraps
+    # around for 5, 10 and 15 of them), in runs that belong to different threads, and whole runs of them
+    for count in (2, 5, 8, 10, 15, 16):
+        X = synth.activations(95, fmt, 1, cols).copy()
+        X[0, 512:512 + count] = np.nan
+        X[0, 1040:1040 + count:2] = np.inf
+        y = _run(fmt, blocks, rows, cols, X, variant)
+        assert not np.isfinite(y).any(), "fmt %d variant %d: %d NaNs in a run were lost" % (fmt, variant, count)
     # the same through a grouped call, and a zero elsewhere in the group does not mask it
     X = np.zeros((1, cols), np.float32)
     X[0, 77] = np.nan
