@@ -93,6 +93,28 @@ def test_outliers_on_zero_weights_stay_inside_the_stated_bound(fmt, variant, zer
     assert worst <= 1.0, "variant %d launched %d: error / bound = %.3g" % (variant, launched, worst)
 
 
+@pytest.mark.parametrize("fmt", [lw.Q8_0, lw.Q4_0])
+def test_tile_kernel_needs_no_extra_term(fmt):
+    # the batched tile kernel decodes every weight exactly before it multiplies: the plain tolerance holds on
+    # the same adversarial activations (eight columns, each with its own outliers), as the header states
+    rows, cols, batch = 48, 4096, 8
+    cols_x = []
+    for b in range(batch):
+        blocks, X = _adversarial(fmt, rows, cols, seed=90 + fmt, zero_rest_of_vector=bool(b & 1))
+        cols_x.append(np.roll(X[0], 0) * (1.0 + b))
+    X = np.stack(cols_x).astype(np.float32)
+    y_ref, s_ref = oracle.matvec(fmt, blocks, rows, cols, X, batch)
+    lw.set_variant(lw.VARIANT_TILE)
+    assert lw.query_variant(fmt, rows, cols, batch) == lw.VARIANT_TILE
+    y = _run(fmt, blocks, rows, cols, X, lw.VARIANT_TILE, batch)
+    worst = float((np.abs(y.astype(np.float64) - y_ref) / (RTOL * s_ref + ATOL)).max())
+    assert worst <= 1.0, "tile kernel: error / tolerance = %.3g" % worst
+    # and a non-finite activation reaches every output of its column only
+    X[3, 100] = np.nan
+    y = _run(fmt, blocks, rows, cols, X, lw.VARIANT_TILE, batch)
+    assert not np.isfinite(y[3]).any() and np.isfinite(np.delete(y, 3, axis=0)).all()
+
+
 @pytest.mark.parametrize("variant", ALL_VARIANTS)
 @pytest.mark.parametrize("fmt", FMTS)
 def test_non_finite_activations_reach_the_output(fmt, variant):
