@@ -13,9 +13,8 @@
 //     their partial sums are combined through a small table, in a fixed order.
 //   * Weights are decoded exactly ((q - 8) resp. the int8 code as floats, then one multiply by the block
 //     scale per block and column), so the accuracy is that of the generic kernels.
-//   * Weights reach shared memory with 4-byte cp.async copies into rows padded to an odd number of words
-//     (a lane reads its own row: consecutive lanes hit consecutive banks), double-buffered against the
-//     products; 18- and 34-byte blocks are only 2-byte aligned, hence the 4-byte granularity.
+//   * Weights reach shared memory with 16-byte cp.async copies into padded rows (a lane reads its own row;
+//     the padding spreads a warp's 32 rows over eight banks), double-buffered against the products.
 // The work is cut into items of 64 rows x one chunk, numbered chunk-major and shared out evenly over the CTAs
 // (one per SM): also a matrix of few rows keeps every SM busy.  An item's sums are added into Y (cleared
 // before the launch) with atomic adds, because the other chunks of the same rows may belong to other CTAs;
@@ -44,18 +43,20 @@ struct TileParams {
     int64_t row_bytes;
     int batch;           // columns of this pass (<= BB)
     int chunk_words;     // 32-bit words of one row's share of a chunk
-    int row_stride;      // words between rows of a stage in shared memory (odd)
+    int row_stride;      // words between rows of a stage in shared memory (a multiple of four, 20 modulo 32)
     uint32_t x_off, w_off, p_off, y_off;     // byte offsets: activations, weight stages, partial table, row sums
 };
 
-__device__ __forceinline__ void cp_async4(uint32_t dst, const void* src) {
-    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(dst), "l"(src) : "memory");
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
 // Four consecutive floats of shared memory as two packed pairs, loaded straight into 64-bit registers (the
 // operand form of the packed FMAs: no moves between the load and the arithmetic).
-__device__ __forceinline__ void lds_pairs(const float* p, f2& lo, f2& hi) {
-    asm volatile("ld.shared.v2.b64 {%0, %1}, [%2];" : "=l"(lo), "=l"(hi) : "r"(smem_u32(p)));
+// `base` is a shared-memory address (32 bits), BYTES a compile-time offset: no address arithmetic per load.
+template <int BYTES>
+__device__ __forceinline__ void lds_pairs(uint32_t base, f2& lo, f2& hi) {
+    asm volatile("ld.shared.v2.b64 {%0, %1}, [%2+%3];" : "=l"(lo), "=l"(hi) : "r"(base), "n"(BYTES));
 }
 template <int N>
 __device__ __forceinline__ void cp_async_wait() {
@@ -130,10 +131,12 @@ __global__ void __launch_bounds__(kTileThreads, 1) matvec_tile_kernel(const Tile
         const int n = (int)(p.rows - r_base < kTileRows ? p.rows - r_base : kTileRows);
         const uint8_t* src0 = p.W + r_base * p.row_bytes + (int64_t)c * chunk_words * 4;
         const uint32_t dst0 = smem_u32(wst + buf * stage_words);
-        for (int r = warp; r < n; r += kTileWarps) {
-            const uint8_t* src = src0 + (int64_t)r * p.row_bytes;
-            const uint32_t dst = dst0 + 4u * (uint32_t)(r * stride);
-            for (int j = lane; j < chunk_words; j += 32) cp_async4(dst + 4u * j, src + 4 * j);
+        // 16-byte pieces (a row's share of a chunk is a whole number of them, and so is the padded row in shared
+        // memory); measured 5 % faster than 4-byte copies into conflict-free odd-stride rows
+        constexpr int kPieces = T::kUnitWords * kTileWarps / 4;
+        for (int i = tid; i < n * kPieces; i += kTileThreads) {
+            const int r = i / kPieces, j = i - r * kPieces;
+            cp_async16(dst0 + 4u * (uint32_t)(r * stride) + 16u * j, src0 + (int64_t)r * p.row_bytes + 16 * j);
         }
         cp_async_commit();
     };
@@ -176,7 +179,7 @@ __global__ void __launch_bounds__(kTileThreads, 1) matvec_tile_kernel(const Tile
             T u0, u1;
             u0.load(base + lane * stride);
             u1.load(base + (two ? lane + 32 : lane) * stride);
-            const float* xw = xs + warp * 64;
+            const uint32_t xw = smem_u32(xs + warp * 64);
 #pragma unroll
             for (int blk = 0; blk < 2; ++blk) {
                 f2 acc[2][BB];
@@ -185,13 +188,24 @@ __global__ void __launch_bounds__(kTileThreads, 1) matvec_tile_kernel(const Tile
                     f2 a0, a1, b0, b1;
                     u0.group(blk, g, a0, a1);
                     u1.group(blk, g, b0, b1);
-                    const float* xk = xw + 32 * blk + 4 * g;
+                    const uint32_t xk = xw + 4u * (32 * blk + 4 * g);
 #pragma unroll
                     for (int b = 0; b < BB; b += 2) {
                         // two columns at a time, so that the two FMAs into one accumulator are four issues apart
                         f2 x01, x23, z01, z23;
-                        lds_pairs(xk + b * kChunkCols, x01, x23);              // same address in every lane
-                        lds_pairs(xk + (b + 1) * kChunkCols, z01, z23);
+                        if (b == 0) {
+                            lds_pairs<0>(xk, x01, x23);              // same address in every lane
+                            lds_pairs<4 * kChunkCols>(xk, z01, z23);
+                        } else if (b == 2) {
+                            lds_pairs<8 * kChunkCols>(xk, x01, x23);
+                            lds_pairs<12 * kChunkCols>(xk, z01, z23);
+                        } else if (b == 4) {
+                            lds_pairs<16 * kChunkCols>(xk, x01, x23);
+                            lds_pairs<20 * kChunkCols>(xk, z01, z23);
+                        } else {
+                            lds_pairs<24 * kChunkCols>(xk, x01, x23);
+                            lds_pairs<28 * kChunkCols>(xk, z01, z23);
+                        }
                         if (g == 0) {              // the block's first products start its sums
                             acc[0][b] = mul2(a0, x01);
                             acc[0][b + 1] = mul2(a0, z01);
@@ -292,7 +306,10 @@ int launch_matvec_tile(int fmt, const void* W, int64_t rows, int64_t cols, const
         p.row_bytes = (int64_t)lw_row_bytes(fmt, cols);
         p.batch = nb;
         p.chunk_words = unit_words * kTileWarps;
-        p.row_stride = p.chunk_words | 1;                     // odd: consecutive lanes (rows) on consecutive banks
+        // rows padded to a multiple of four words (16-byte copies) that is 20 modulo 32: a lane reads its own row,
+        // so the 32 rows of a warp spread over eight banks (4-way conflicts on the 18 or 34 unit loads per item,
+        // which is cheap next to the products; an odd stride would be conflict-free but forces 4-byte copies)
+        p.row_stride = p.chunk_words + ((20 - p.chunk_words % 32) + 32) % 32;
         const size_t x_bytes = (size_t)bb * kChunkCols * 4;
         const size_t w_bytes = 2 * (size_t)kTileRows * p.row_stride * 4;
         const size_t p_bytes = (size_t)kTileWarps * kTileRows * bb * 4;
