@@ -103,8 +103,10 @@ int lw_dequant(int fmt, const void* W_blocks, int64_t n, float* out, void* strea
 
 /* Fused dequantise + mat-vec [Sec 3.2, 3.3]: Y[b*rows + r] = sum_k decode(W)[r][k] * X[b*cols + k],
  * fp32 accumulation, for b < batch (1..16).  The batched kernels reuse every decoded block for all
- * their columns; without a forced variant the quantised formats (and f16 up to four columns) run one
- * streaming pass per column instead (four columns per launch), which measures faster on B200.
+ * their columns: without a forced variant q8_0 and q4_0 with cols a multiple of 256 run on the tensor
+ * cores from three columns on (LW_VARIANT_MMA); the other quantised formats (and f16 up to four columns)
+ * run one streaming pass per column instead (four columns per launch), which measures faster on B200
+ * than their batched kernels.
  * W_blocks: device, rows * lw_row_bytes(fmt, cols) bytes, row-major without padding, 16-byte
  *           aligned, read-only.
  * X: device, batch * cols floats, each activation vector contiguous, 16-byte aligned, read-only.
@@ -113,7 +115,9 @@ int lw_dequant(int fmt, const void* W_blocks, int64_t n, float* out, void* strea
  * Accuracy.  With w the decoded weights and S = sum_k |w_k x_k|, every result satisfies
  *     |y - y_exact| <= 1e-4 * S + 1e-6 + E .
  * E = 0 for LW_VARIANT_GENERIC and for f16 (each weight is decoded exactly and then multiplied: plain fp32
- * accumulation), for any finite input.  The streaming variants multiply the integer codes first and apply
+ * accumulation), for any finite input, and for the batched LW_VARIANT_TILE and LW_VARIANT_MMA (exact integer
+ * codes times exact activations, block sums scaled in fp32) as long as |x| <= 2^115, which keeps a block's
+ * sum of code * x finite.  The streaming variants multiply the integer codes first and apply
  * block scales and offsets to the sums, and LW_VARIANT_IDOT holds the activations as block fixed point
  * (23 bits + sign relative to the largest magnitude in each run of 16 or 32), so an activation that is
  * huge compared with its neighbours and meets a weight that is zero or nearly so leaves an absolute error
@@ -218,18 +222,25 @@ typedef enum {
                                statement of lw_matvec).  All nine quantised formats (f16 falls back to
                                LW_VARIANT_STREAM).  q8_0, q4_0 and q4_K also have a batched form (2..16
                                columns, fixed-point activations kept in shared memory) */
-    LW_VARIANT_TILE = 4     /* batch 2..16 only: fp32 tile kernel, a lane owns rows, every weight is decoded once
+    LW_VARIANT_TILE = 4,    /* batch 2..16 only: fp32 tile kernel, a lane owns rows, every weight is decoded once
                                (exactly) and multiplied with all columns of a pass (up to 8) by packed fp32 FMAs,
                                activations read from shared memory by broadcast; q8_0 and q4_0, cols a multiple
                                of 1024.  E = 0 in the accuracy statement of lw_matvec; a row's sum is completed
                                with atomic additions (one per 1024 columns), so the last bits of a result can
-                               differ from run to run.  AUTO takes it from 7 columns on (passes of 7 or 8 columns;
-                               a remainder of fewer goes through the batch-1 kernel column by column) */
+                               differ from run to run.  Not chosen by AUTO (LW_VARIANT_MMA covers its shapes and
+                               is faster); forced, it runs passes of 8 and 4 columns */
+    LW_VARIANT_MMA = 5      /* batch 2..16 only: tensor-core kernel (mma m16n8k16, bf16 operands, fp32 accumulation).
+                               A weight's integer code is exact in bf16 and the block scale is applied in fp32 to each
+                               block's sum; every fp32 activation is cut into three bf16 terms that add up to it
+                               exactly, so E = 0 in the accuracy statement of lw_matvec.  q8_0 and q4_0, cols a
+                               multiple of 256; all columns in one pass over the weights.  A row's sum is completed
+                               with atomic additions (one per chunk of up to 1024 columns), so the last bits of a
+                               result can differ from run to run.  AUTO takes it from 3 columns on */
 } lw_variant;
 /* Process-wide; returns LW_ERR_FORMAT for an unknown value.  Also settable once at load time
  * through the environment variable LW_FORCE_VARIANT (a number).  A forced variant that does not
  * support the problem (shape, batch, format) falls back to the next simpler one.  AUTO picks, when
- * the shape qualifies: IDOT for the quantised formats (batch 2..16: TILE from 7 columns on where it applies,
+ * the shape qualifies: IDOT for the quantised formats (batch 3..16: MMA where it applies,
  * else IDOT's batch-1 kernel once per column), STREAM for f16 up to batch 4 (likewise); otherwise GENERIC. */
 int lw_set_variant(int variant);
 /* The variant lw_matvec would launch for this problem (after forcing and shape checks), or a

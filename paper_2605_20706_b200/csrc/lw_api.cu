@@ -18,7 +18,7 @@ static int forced_variant() {
     v = LW_VARIANT_AUTO;
     if (const char* env = std::getenv("LW_FORCE_VARIANT")) {
         const int e = std::atoi(env);
-        if (e >= LW_VARIANT_AUTO && e <= LW_VARIANT_TILE) v = e;
+        if (e >= LW_VARIANT_AUTO && e <= LW_VARIANT_MMA) v = e;
     }
     int expected = -1;
     g_variant.compare_exchange_strong(expected, v);
@@ -43,6 +43,7 @@ static int check_matvec_args(int fmt, const void* W, int64_t rows, int64_t cols,
 // but 2.69 / 5.32 ms against 2.19 / 4.51 ms at batch 8 / 16.
 constexpr int kColumnsPerLaunch = 4;
 constexpr int kTileMinColumns = 7;
+constexpr int kMmaMinColumns = 3;
 static bool columnwise(int fmt, int64_t rows, int64_t cols, int batch) {
     if (fmt == LW_F16 && batch > 4) return false;      // f16 from 5 columns: the tiled fp32 kernel is faster
     return batch > 1 && forced_variant() == LW_VARIANT_AUTO && rows <= INT32_MAX &&
@@ -52,10 +53,14 @@ static bool columnwise(int fmt, int64_t rows, int64_t cols, int batch) {
 
 static int pick_variant(int fmt, int64_t rows, int64_t cols, int batch) {
     const int forced = forced_variant();
-    // batch 2..16: the fp32 tile kernel where it applies (every decoded weight is used for all columns of a
-    // pass).  Measured on the 8B shapes (ms per step, q4_0): a pass of 8 columns 6.0, of 4 columns 4.2, against
-    // 2.2 / 3.7 / 7.3 for 2 / 4 / 8 columns through the batch-1 kernel: AUTO takes it from seven columns on, in
-    // passes of seven or eight, and leaves a remainder of fewer columns to the batch-1 kernel.
+    // batch 2..16: the tensor-core kernel where it applies (q8_0 / q4_0, cols a multiple of 256; all columns in one
+    // pass over the weights).  Measured on the 8B shapes (ms per step, q4_0): 2.6 / 2.65 / 2.7 / 3.7 for 2 / 4 / 8 /
+    // 16 columns, against 2.2 / 3.7 / 7.3 for 2 / 4 / 8 columns through the batch-1 kernel and 6.0 / 11.6 for 8 / 16
+    // through the fp32 tile kernel: AUTO takes it from three columns on.  The fp32 tile kernel stays for forced
+    // selection (and for AUTO where only it applies: never, today -- its shapes are a subset).
+    if (matvec_mma_supported(fmt, rows, cols, batch) &&
+        (forced == LW_VARIANT_MMA || (forced == LW_VARIANT_AUTO && batch >= kMmaMinColumns)))
+        return LW_VARIANT_MMA;
     if (matvec_tile_supported(fmt, rows, cols, batch) &&
         (forced == LW_VARIANT_TILE || (forced == LW_VARIANT_AUTO && batch >= kTileMinColumns)))
         return LW_VARIANT_TILE;
@@ -153,7 +158,9 @@ int lw_matvec(int fmt, const void* W_blocks, int64_t rows, int64_t cols, const f
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     int err;
     const int variant = pick_variant(fmt, rows, cols, batch);
-    if (variant == LW_VARIANT_TILE && forced_variant() == LW_VARIANT_AUTO) {
+    if (variant == LW_VARIANT_MMA) {
+        err = launch_matvec_mma(fmt, W_blocks, rows, cols, X, Y, batch, s);
+    } else if (variant == LW_VARIANT_TILE && forced_variant() == LW_VARIANT_AUTO) {
         // passes of seven or eight columns through the tile kernel, the remainder through the batch-1 kernel
         const int tiled = batch - (batch % 8 >= kTileMinColumns ? 0 : batch % 8);
         err = launch_matvec_tile(fmt, W_blocks, rows, cols, X, Y, tiled, s);
@@ -337,7 +344,7 @@ int lw_matvec_host(int fmt, const void* W_blocks, int64_t rows, int64_t cols, co
 }
 
 int lw_set_variant(int variant) {
-    if (variant < LW_VARIANT_AUTO || variant > LW_VARIANT_TILE) return LW_ERR_FORMAT;
+    if (variant < LW_VARIANT_AUTO || variant > LW_VARIANT_MMA) return LW_ERR_FORMAT;
     g_variant.store(variant);
     return LW_OK;
 }

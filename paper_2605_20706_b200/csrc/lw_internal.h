@@ -48,6 +48,11 @@ int launch_probe_read(const void* src, int64_t bytes, cudaStream_t stream);
 bool matvec_tile_supported(int fmt, int64_t rows, int64_t cols, int batch);
 int launch_matvec_tile(int fmt, const void* W, int64_t rows, int64_t cols, const float* X, float* Y, int batch,
                        cudaStream_t stream);
+// Batched tensor-core kernel (2..16 columns; weights as exact bf16 codes, activations as three bf16 terms, fp32
+// accumulation): q8_0 and q4_0 with cols a multiple of 256.  The launch clears Y first (the kernel adds into it).
+bool matvec_mma_supported(int fmt, int64_t rows, int64_t cols, int batch);
+int launch_matvec_mma(int fmt, const void* W, int64_t rows, int64_t cols, const float* X, float* Y, int batch,
+                      cudaStream_t stream);
 // Tunables of the streaming kernels (0 = automatic) and the geometry they lead to for a shape.
 void set_stream_tuning(int worker_groups, int stages, int stage_kb);
 // Per-shape tunables (all zero erases the entry); make_plan uses them where the process-wide ones are 0.

@@ -1,0 +1,551 @@
+// Batched mat-vec on the tensor cores (batch 2..16, q4_0 and q8_0) [paper Sec 3.2: from a handful of columns on
+// the mat-vec turns into a small mat-mat product, a dense contraction; Sec 3.3: one decode routine per format
+// spliced into a common skeleton].
+//
+// With several columns the products, not the weight bytes, bound an fp32 kernel (74 TFLOP/s of packed FMAs at
+// best, against the 98 / 196 TFLOP/s that 8 / 16 columns need to keep up with the weight stream of q4_0).  This
+// kernel computes Y[b][r] = sum_k W[r][k] X[b][k] with mma.sync.m16n8k16 (bf16 x bf16 -> f32) and loses nothing
+// to the narrow operand type:
+//   * the integer code of a weight (q - 8 in [-8, 7], resp. an int8) is exact in bf16; the fp16 block scale is
+//     applied in fp32 to each block's sum, as in the definition;
+//   * an fp32 activation is cut into three bf16 terms of eight significant bits each, by truncation:
+//     x = x1 + x2 + x3 exactly, so that code * x1 + code * x2 + code * x3, accumulated in fp32 by the tensor
+//     core, is the fp32-accumulated product with the exact activation.  A NaN or Inf stays one (in x1 or x2).
+// The accuracy is therefore that of the fp32 kernels: |y - y_ref| <= 1e-4 * sum|w x| + 1e-6 with no extra term.
+//
+// Why mma.sync and not tcgen05.mma here: the A operand is the decoded weight, which exists only in registers
+// (18- and 34-byte blocks decode to fragments with byte permutes); tcgen05.mma reads A from shared or tensor
+// memory, so every weight would take one more store and a proxy fence, for an N of 8..48 whose tensor time is
+// already far below the decode time.  The warp-level form takes the fragments straight from the decode.
+//
+// Layout of the work.  A stage is 256 rows x 256 columns of weights (36 KB of q4_0, 68 KB of q8_0), brought in
+// by a producer thread with one tiled bulk-tensor copy (the matrix as a 2-D tensor of 32-bit words; rows beyond
+// the matrix arrive as zeros) into a ring of stages (full / empty mbarriers).  One 1-D bulk copy per row piece
+// was measured at about 40 ns per copy, 10 us per stage.
+// Each of 16 compute warps owns 16 rows of the stage (the M of the mma) and walks the stage's four 64-weight
+// units; a lane (g = lane / 4, t = lane % 4) reads word t of the quants of rows g and g + 8, which holds
+// exactly the eight weights of its A fragments once the k index inside a block is permuted -- the same
+// permutation is applied to the activations when a lane loads its B fragments, and a sum does not care.
+// The activations of a chunk of up to 1024 columns sit in shared memory as three bf16 planes.  Stages are
+// numbered chunk-major, (row stage, sub-stage)-minor and dealt out in equal contiguous ranges to one CTA per
+// SM, so a matrix of few rows still keeps every SM busy; sums stay in registers while a CTA stays inside one
+// (chunk, row stage) and are then added into Y, which the host clears before the launch, with atomic adds
+// (the other chunks of the same rows may belong to other CTAs).  The order of those adds is not fixed: results
+// may differ in the last bits from run to run, within the tolerance.
+//
+// All waits are bounded: a wait that gives up records a fault code, the CTA stops waiting and copying, the
+// producer drains what it has in flight, and the kernel terminates (its results are then meaningless and
+// lw_device_status reports the fault).
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <cstdint>
+
+#include "lw.h"
+#include "lw_internal.h"
+#include "lw_stream_common.cuh"
+
+namespace lw {
+namespace {
+
+constexpr int kMmaWarps = 16;                         // compute warps
+constexpr int kMmaComputeThreads = 32 * kMmaWarps;
+constexpr int kMmaThreads = kMmaComputeThreads + 32;  // plus the producer warp
+constexpr int kStageRows = 16 * kMmaWarps;            // 256
+constexpr int kStageCols = 256;
+constexpr int kStageUnits = kStageCols / 64;
+constexpr int kMaxRing = 4;
+constexpr int kXPad = 64;                             // bytes after each column of a plane: 16-byte loads of lanes
+                                                      // (g, t) at 64 g + 16 t cover 128 distinct bytes per quarter warp
+constexpr int kMmaHeader = 128;                       // barriers and the stop flag
+
+struct MmaParams {
+    const uint8_t* W;
+    const float* X;
+    float* Y;
+    int* fault;
+    int64_t rows, cols, row_bytes;
+    int batch;            // columns of this launch (<= 8 NT)
+    int chunk_cols;       // 256, 512 or 1024: columns whose activations are resident at a time
+    int ring;             // stages in the ring (2..kMaxRing)
+    uint32_t x_off, w_off;
+};
+
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void compute_barrier() {
+    asm volatile("bar.sync 1, %0;" ::"n"(kMmaComputeThreads) : "memory");
+}
+__device__ __forceinline__ uint32_t sub_bf16x2(uint32_t a, uint32_t b) {
+    uint32_t d;
+    asm("sub.rn.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
+// Shared-memory loads at `base` + a compile-time byte offset: no address arithmetic per load.
+template <int OFF>
+__device__ __forceinline__ uint32_t lds32(uint32_t base) {
+    uint32_t v;
+    asm volatile("ld.shared.b32 %0, [%1+%2];" : "=r"(v) : "r"(base), "n"(OFF));
+    return v;
+}
+template <int OFF>
+__device__ __forceinline__ float lds_half(uint32_t base) {
+    unsigned short h;
+    asm volatile("ld.shared.u16 %0, [%1+%2];" : "=h"(h) : "r"(base), "n"(OFF));
+    return __half2float(__ushort_as_half(h));
+}
+template <int OFF>
+__device__ __forceinline__ void lds128(uint32_t base, uint32_t& a, uint32_t& b, uint32_t& c, uint32_t& d) {
+    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4+%5];" : "=r"(a), "=r"(b), "=r"(c), "=r"(d) : "r"(base), "n"(OFF));
+}
+// D = A (16 x 16, row) * B (16 x 8, col) + D, bf16 operands, fp32 accumulators
+__device__ __forceinline__ void mma_bf16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                         uint32_t b1) {
+    asm("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+        "{%0, %1, %2, %3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+// The same with D = A * B (the first product of a sum)
+__device__ __forceinline__ void mma_bf16_first(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                               uint32_t b0, uint32_t b1) {
+    asm("{\n\t.reg .f32 z;\n\tmov.f32 z, 0f00000000;\n\t"
+                 "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+                 "{z, z, z, z};\n\t}"
+                 : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+// One box of the 2-D tensor behind `map` (x = first 32-bit word of the row piece, y = first row) into shared
+// memory at `dst` (128-byte aligned); completion is counted in bytes on `bar`.  x * 4 must be a multiple of 16.
+__device__ __forceinline__ void tensor_load_2d(void* dst, const CUtensorMap* map, int x, int y, uint64_t* bar,
+                                               uint64_t policy) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes.L2::cache_hint "
+        "[%0], [%1, {%2, %3}], [%4], %5;" ::"r"(smem_u32(dst)),
+        "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(smem_u32(bar)), "l"(policy)
+        : "memory");
+}
+
+// Two bytes of `v` (I and I + 1) as the bf16 pair (128 + byte I, 128 + byte I + 1): each byte lands in the seven
+// mantissa bits of 128.0 (0x4300), so it must be below 128.
+template <int I>
+__device__ __forceinline__ uint32_t bytes_to_bf16_128_plus(uint32_t v) {
+    return __byte_perm(v, 0x43434343u, I == 0 ? 0x4140u : 0x4342u);
+}
+
+// A lane's weights of one block of one row: four bf16 pairs.  p[0], p[1] = weights 4t .. 4t+3 of the block,
+// p[2], p[3] = weights 16+4t .. 16+4t+3 (the k order the B fragments follow).  `wt` = shared-memory address of
+// the row's piece of the stage plus 4 t (t = lane % 4), OFF = byte offset of the two-block unit from there.
+struct MmaQ40 {
+    static constexpr int kBlockBytes = 18;
+    template <int OFF, int BLK>
+    static __device__ __forceinline__ void block(uint32_t wt, uint32_t (&p)[4]) {
+        uint32_t q;
+        if (BLK == 0)                                   // quants at bytes 2..17: word t straddles two words
+            q = __byte_perm(lds32<OFF>(wt), lds32<OFF + 4>(wt), 0x5432u);
+        else                                            // quants at bytes 20..35
+            q = lds32<OFF + 20>(wt);
+        const uint32_t lo = q & 0x0F0F0F0Fu, hi = (q >> 4) & 0x0F0F0F0Fu;
+        const uint32_t bias = 0x43084308u;              // (136, 136): (128 + q) - 136 = q - 8, exactly
+        p[0] = sub_bf16x2(bytes_to_bf16_128_plus<0>(lo), bias);
+        p[1] = sub_bf16x2(bytes_to_bf16_128_plus<2>(lo), bias);
+        p[2] = sub_bf16x2(bytes_to_bf16_128_plus<0>(hi), bias);
+        p[3] = sub_bf16x2(bytes_to_bf16_128_plus<2>(hi), bias);
+    }
+    // `row` = address of the row's piece (without the lane's 4 t)
+    template <int OFF, int BLK>
+    static __device__ __forceinline__ float scale(uint32_t row) { return lds_half<OFF + 18 * BLK>(row); }
+};
+
+struct MmaQ80 {
+    static constexpr int kBlockBytes = 34;
+    // An int8 code c as bf16: 0x4300 | (c & 0x7F) is 128 + (c & 0x7F), and 0x4300 | (c & 0x80) is 128 or 256;
+    // their difference is c.
+    static __device__ __forceinline__ uint32_t pair(uint32_t v) {
+        return sub_bf16x2(v & 0xFF7FFF7Fu, v & 0xFF80FF80u);
+    }
+    template <int OFF, int BLK>
+    static __device__ __forceinline__ void block(uint32_t wt, uint32_t (&p)[4]) {
+        uint32_t qa, qb;                                // quant words t and 4 + t of the block
+        if (BLK == 0) {                                 // quants at bytes 2..33
+            qa = __byte_perm(lds32<OFF>(wt), lds32<OFF + 4>(wt), 0x5432u);
+            qb = __byte_perm(lds32<OFF + 16>(wt), lds32<OFF + 20>(wt), 0x5432u);
+        } else {                                        // quants at bytes 36..67
+            qa = lds32<OFF + 36>(wt);
+            qb = lds32<OFF + 52>(wt);
+        }
+        p[0] = pair(__byte_perm(qa, 0x43434343u, 0x4140u));
+        p[1] = pair(__byte_perm(qa, 0x43434343u, 0x4342u));
+        p[2] = pair(__byte_perm(qb, 0x43434343u, 0x4140u));
+        p[3] = pair(__byte_perm(qb, 0x43434343u, 0x4342u));
+    }
+    template <int OFF, int BLK>
+    static __device__ __forceinline__ float scale(uint32_t row) { return lds_half<OFF + 34 * BLK>(row); }
+};
+
+// One block (32 weights) of the warp's 16 rows against all columns: decode the lane's fragments of rows g and
+// g + 8, six products per group of eight columns into one accumulator, then the block scales in fp32.
+// U = unit of the stage (0..3), BLK = block of the unit; xp[nt][s] = address of the lane's B fragments of plane s,
+// column group nt, at the stage's first column.
+template <class T, int NT, int U, int BLK>
+__device__ __forceinline__ void block_step(uint32_t wt, uint32_t row, const uint32_t (&xp)[NT][3], float (&y)[NT][4]) {
+    constexpr int kPiece = kStageCols / 32 * T::kBlockBytes;
+    constexpr int kUnit = U * 2 * T::kBlockBytes;
+    uint32_t a[4], b[4];
+    T::template block<kUnit, BLK>(wt, a);
+    T::template block<kUnit + 8 * kPiece, BLK>(wt, b);
+    const float d0 = T::template scale<kUnit, BLK>(row), d1 = T::template scale<kUnit + 8 * kPiece, BLK>(row);
+    constexpr int kX = 2 * (64 * U + 32 * BLK);          // bytes into a plane's column
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+        float c[4];
+#pragma unroll
+        for (int s = 0; s < 3; ++s) {
+            uint32_t b0, b1, b2, b3;
+            lds128<kX>(xp[nt][s], b0, b1, b2, b3);      // k = 4t .. 4t+3 and k = 16+4t .. 16+4t+3
+            if (s == 0)
+                mma_bf16_first(c, a[0], b[0], a[1], b[1], b0, b1);
+            else
+                mma_bf16(c, a[0], b[0], a[1], b[1], b0, b1);
+            mma_bf16(c, a[2], b[2], a[3], b[3], b2, b3);
+        }
+        y[nt][0] = fmaf(d0, c[0], y[nt][0]);
+        y[nt][1] = fmaf(d0, c[1], y[nt][1]);
+        y[nt][2] = fmaf(d1, c[2], y[nt][2]);
+        y[nt][3] = fmaf(d1, c[3], y[nt][3]);
+    }
+}
+
+// fp32 -> three bf16 terms by truncation (x1 + x2 + x3 == x exactly; the differences are exact in fp32)
+__device__ __forceinline__ void split3(float x, uint32_t& h1, uint32_t& h2, uint32_t& h3) {
+    const uint32_t b1 = __float_as_uint(x) & 0xFFFF0000u;
+    const float r1 = x - __uint_as_float(b1);
+    const uint32_t b2 = __float_as_uint(r1) & 0xFFFF0000u;
+    const float r2 = r1 - __uint_as_float(b2);
+    h1 = b1 >> 16;
+    h2 = b2 >> 16;
+    h3 = __float_as_uint(r2) >> 16;                     // at most eight significant bits are left: exact
+}
+
+// Where a CTA is in its range of stages: chunk c, row stage rs, sub-stage j of the chunk, ring slot and the
+// parity of the slot's current use.  Stepped without divisions.
+struct Cursor {
+    int c, rs, j, slot;
+    uint32_t parity;
+    __device__ __forceinline__ void init(int64_t first, int spc, int n_rs) {
+        const int64_t pair = first / spc;
+        j = (int)(first - pair * spc);
+        c = (int)(pair / n_rs);
+        rs = (int)(pair - (int64_t)c * n_rs);
+        slot = 0;
+        parity = 0;
+    }
+    __device__ __forceinline__ void step(int spc, int n_rs, int ring) {
+        if (++slot == ring) {
+            slot = 0;
+            parity ^= 1u;
+        }
+        if (++j == spc) {
+            j = 0;
+            if (++rs == n_rs) {
+                rs = 0;
+                ++c;
+            }
+        }
+    }
+};
+
+template <class T, int NT>
+__global__ void __launch_bounds__(kMmaThreads, 1) matvec_mma_kernel(const __grid_constant__ MmaParams p,
+                                                                    const __grid_constant__ CUtensorMap wmap) {
+    extern __shared__ __align__(128) uint8_t smem[];
+    uint64_t* full = reinterpret_cast<uint64_t*>(smem);               // [kMaxRing]
+    uint64_t* empty = full + kMaxRing;                                // [kMaxRing]
+    volatile int* stop = reinterpret_cast<volatile int*>(smem + 64);  // set when a wait gave up
+    constexpr int NB = 8 * NT;                                        // columns held (beyond the batch: zeros)
+    constexpr int kPiece = kStageCols / 32 * T::kBlockBytes;          // bytes of a row's share of a stage
+    constexpr int kStageBytes = kStageRows * kPiece;
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int Kx = p.chunk_cols;
+    const uint32_t x_pitch = 2u * Kx + kXPad;                         // bytes between columns of a plane
+    const uint32_t plane_pitch = NB * x_pitch;
+    const int spc = Kx / kStageCols;                                  // stages per (chunk, row stage)
+    const int n_rs = (int)((p.rows + kStageRows - 1) / kStageRows);
+    const int n_chunks = (int)(p.cols / Kx);
+    const int64_t n_stages = (int64_t)n_chunks * n_rs * spc;
+    const int64_t first = n_stages * blockIdx.x / gridDim.x, last = n_stages * (blockIdx.x + 1) / gridDim.x;
+    const int ring = p.ring;
+
+    if (tid == 0) {
+        for (int s = 0; s < kMaxRing; ++s) {
+            mbar_init(&full[s], 1);
+            mbar_init(&empty[s], kMmaWarps);
+        }
+        *stop = 0;
+        fence_barrier_init();
+    }
+    __syncthreads();
+
+    if (warp == kMmaWarps) {
+        // ------------------------------------------------------------- producer (one thread) ---
+        if (lane != 0) return;
+        const uint64_t policy = l2_evict_first_policy();
+        const int count = (int)(last - first);
+        Cursor cur;
+        cur.init(first, spc, n_rs);
+        int n = 0;
+        for (; n < count; ++n, cur.step(spc, n_rs, ring)) {
+            if (*stop) break;
+            if (n >= ring && !mbar_wait_bounded(&empty[cur.slot], cur.parity ^ 1u)) {   // the slot's previous use
+                atomicExch(p.fault, (int)FAULT_BULK_WAIT_TIMEOUT);
+                *stop = 1;
+                break;
+            }
+            mbar_expect_tx(&full[cur.slot], kStageBytes);   // a box always delivers all its bytes (zeros past the end)
+            tensor_load_2d(smem + p.w_off + (size_t)cur.slot * kStageBytes, &wmap, (cur.c * spc + cur.j) * (kPiece / 4),
+                           cur.rs * kStageRows, &full[cur.slot], policy);
+        }
+        if (*stop) {
+            // the consumers have stopped waiting: make sure nothing is still landing in shared memory (stage m,
+            // the latest armed use of its slot, is the (m / ring)-th use)
+            for (int m = n - 1; m >= 0 && m >= n - ring; --m)
+                if (!mbar_wait_bounded(&full[m % ring], (uint32_t)(m / ring) & 1u))
+                    atomicExch(p.fault, (int)FAULT_DRAIN_TIMEOUT);
+        }
+        return;
+    }
+
+    // ------------------------------------------------------------------- compute warps ---
+    const int g = lane >> 2, t = lane & 3;
+    const uint32_t xs = smem_u32(smem + p.x_off);
+    // this lane's B fragments: column g of each group of eight, slots 8 t .. 8 t + 7 of a block of 32
+    const uint32_t xlane = xs + g * x_pitch + 16u * t;
+    const uint32_t wrow = smem_u32(smem + p.w_off) + (uint32_t)(16 * warp + g) * kPiece;   // row g of this warp's 16
+
+    float y[NT][4];
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) y[nt][i] = 0.f;
+    int cur_c = -1, cur_rs = -1;
+
+    auto flush = [&]() {
+        // add this warp's sums of (chunk, row stage cur_rs) into Y: rows g and g + 8 of the warp's 16, columns
+        // 8 nt + 2 t and 8 nt + 2 t + 1
+        const int64_t r = (int64_t)cur_rs * kStageRows + 16 * warp + g;
+#pragma unroll
+        for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const int b = 8 * nt + 2 * t + (i & 1);
+                const int64_t rr = r + (i >> 1) * 8;
+                if (b < p.batch && rr < p.rows) atomicAdd(p.Y + (int64_t)b * p.rows + rr, y[nt][i]);
+                y[nt][i] = 0.f;
+            }
+    };
+
+    const int count = (int)(last - first);
+    Cursor cur;
+    cur.init(first, spc, n_rs);
+    for (int n = 0; n < count; ++n, cur.step(spc, n_rs, ring)) {
+        const int c = cur.c, rs = cur.rs, j = cur.j, slot = cur.slot;
+        if (c != cur_c || rs != cur_rs) {
+            if (cur_rs >= 0) flush();
+            cur_rs = rs;
+        }
+        if (c != cur_c) {
+            // the chunk's activations as three bf16 planes: plane s, column b.  Inside a block of 32 the order is
+            // the one the fragments want: slots 8 q .. 8 q + 3 hold k = 4 q .. 4 q + 3 and slots 8 q + 4 .. 8 q + 7
+            // hold k = 16 + 4 q .., so a lane reads both halves of its B operand with one 16-byte load.
+            cur_c = c;
+            compute_barrier();                          // every warp is done with the previous chunk
+            // Only the 256-column pieces this CTA's stages inside the chunk will read (all of them once it has
+            // `spc` or more stages here); a piece is 64 quads of each column: one quad per thread and group of
+            // eight columns.  All loads are issued before the first conversion.
+            const int64_t in_chunk = (int64_t)(n_rs - rs) * spc - j;
+            const int left = count - n;
+            const int m = (int)(in_chunk < left ? in_chunk : left);
+            float4 v[4][NT];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const int jj = (j + q) % spc;
+#pragma unroll
+                for (int nt = 0; nt < NT; ++nt) {
+                    const int b = 8 * nt + (tid >> 6), k4 = jj * (kStageCols / 4) + (tid & 63);
+                    v[q][nt] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (q < spc && q < m && b < p.batch)
+                        v[q][nt] = __ldg(reinterpret_cast<const float4*>(p.X + (int64_t)b * p.cols + (int64_t)c * Kx) + k4);
+                }
+            }
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const int jj = (j + q) % spc;
+                if (q < spc && q < m) {
+#pragma unroll
+                    for (int nt = 0; nt < NT; ++nt) {
+                        const int b = 8 * nt + (tid >> 6), k4 = jj * (kStageCols / 4) + (tid & 63);
+                        uint32_t h[3][4];
+                        split3(v[q][nt].x, h[0][0], h[1][0], h[2][0]);
+                        split3(v[q][nt].y, h[0][1], h[1][1], h[2][1]);
+                        split3(v[q][nt].z, h[0][2], h[1][2], h[2][2]);
+                        split3(v[q][nt].w, h[0][3], h[1][3], h[2][3]);
+                        const int slot4 = (k4 & ~7) + 2 * (k4 & 3) + ((k4 >> 2) & 1);    // quad of slots the quad of k goes to
+                        const uint32_t dst = xs + b * x_pitch + 8u * slot4;
+#pragma unroll
+                        for (int s = 0; s < 3; ++s)
+                            asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(dst + s * plane_pitch),
+                                         "r"(h[s][0] | (h[s][1] << 16)), "r"(h[s][2] | (h[s][3] << 16))
+                                         : "memory");
+                    }
+                }
+            }
+            compute_barrier();
+        }
+        if (!*stop && !mbar_wait_bounded(&full[slot], cur.parity)) {
+            if (lane == 0) {
+                atomicExch(p.fault, (int)FAULT_BULK_WAIT_TIMEOUT);
+                *stop = 1;
+            }
+        }
+        const int64_t r0 = (int64_t)rs * kStageRows;
+        if (r0 + 16 * warp < p.rows) {
+            const uint32_t row = wrow + (uint32_t)slot * kStageBytes, wt = row + 4u * t;
+            uint32_t xp[NT][3];
+#pragma unroll
+            for (int nt = 0; nt < NT; ++nt)
+#pragma unroll
+                for (int s = 0; s < 3; ++s)
+                    xp[nt][s] = xlane + 2u * (uint32_t)(j * kStageCols) + s * plane_pitch + nt * 8 * x_pitch;
+            block_step<T, NT, 0, 0>(wt, row, xp, y);
+            block_step<T, NT, 0, 1>(wt, row, xp, y);
+            block_step<T, NT, 1, 0>(wt, row, xp, y);
+            block_step<T, NT, 1, 1>(wt, row, xp, y);
+            block_step<T, NT, 2, 0>(wt, row, xp, y);
+            block_step<T, NT, 2, 1>(wt, row, xp, y);
+            block_step<T, NT, 3, 0>(wt, row, xp, y);
+            block_step<T, NT, 3, 1>(wt, row, xp, y);
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&empty[slot]);
+    }
+    if (cur_rs >= 0) flush();
+}
+
+template <class T, int NT>
+int launch_mma(const MmaParams& p, const CUtensorMap& wmap, int grid, size_t smem_bytes, cudaStream_t stream) {
+    static bool attr_set[64] = {false};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return (int)e;
+    if (dev < 0 || dev >= 64 || !attr_set[dev]) {
+        e = cudaFuncSetAttribute(matvec_mma_kernel<T, NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        if (e != cudaSuccess) return (int)e;
+        if (dev >= 0 && dev < 64) attr_set[dev] = true;
+    }
+    matvec_mma_kernel<T, NT><<<(unsigned)grid, kMmaThreads, smem_bytes, stream>>>(p, wmap);
+    return (int)cudaGetLastError();
+}
+
+// cuTensorMapEncodeTiled through the runtime's driver entry point lookup (no link against the driver library)
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn encode_tiled_fn() {
+    static EncodeTiledFn fn = [] {
+        void* f = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess)
+            f = nullptr;
+        return reinterpret_cast<EncodeTiledFn>(f);
+    }();
+    return fn;
+}
+
+// The weight matrix as a 2-D tensor of 32-bit words (row_bytes / 4 per row, `rows` rows) with boxes of one stage.
+bool make_weight_map(CUtensorMap* map, const void* W, int64_t rows, int64_t row_bytes, int piece_bytes) {
+    EncodeTiledFn fn = encode_tiled_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)(row_bytes / 4), (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)row_bytes};
+    const cuuint32_t box[2] = {(cuuint32_t)(piece_bytes / 4), (cuuint32_t)kStageRows};
+    const cuuint32_t elem[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<void*>(W), dims, strides, box, elem,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+int mma_sm_count() {
+    int dev = 0, n = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return 148;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) return 148;
+    return n;
+}
+
+// Shared-memory plan of a launch: the largest chunk (1024, 512, 256 columns) that divides cols and leaves room
+// for at least two stages.  Returns false if nothing fits.
+bool mma_plan(int fmt, int64_t cols, int nt, int& chunk_cols, int& ring, size_t& x_bytes, size_t& stage_bytes) {
+    const int block_bytes = fmt == LW_Q4_0 ? 18 : 34;
+    stage_bytes = (size_t)kStageRows * (kStageCols / 32) * block_bytes;
+    const size_t budget = 227 * 1024 - kMmaHeader;
+    for (int kx = 1024; kx >= 256; kx /= 2) {
+        if (cols % kx != 0) continue;
+        x_bytes = (size_t)3 * 8 * nt * (2 * kx + kXPad);
+        if (x_bytes + 2 * stage_bytes > budget) continue;
+        size_t n = (budget - x_bytes) / stage_bytes;
+        ring = (int)(n > (size_t)kMaxRing ? kMaxRing : n);
+        chunk_cols = kx;
+        return true;
+    }
+    return false;
+}
+
+}  // namespace
+
+bool matvec_mma_supported(int fmt, int64_t rows, int64_t cols, int batch) {
+    if (fmt != LW_Q4_0 && fmt != LW_Q8_0) return false;
+    if (batch < 2 || batch > 16) return false;
+    if (cols % kStageCols != 0) return false;
+    return rows >= 1 && rows <= (int64_t)1 << 30;
+}
+
+// Arguments are validated by the caller; returns a cudaError_t as int.
+int launch_matvec_mma(int fmt, const void* W, int64_t rows, int64_t cols, const float* X, float* Y, int batch,
+                      cudaStream_t stream) {
+    int* fault = device_fault_word();
+    if (!fault) return (int)cudaErrorInvalidValue;
+    // the kernel adds every (chunk, row stage) share into Y
+    cudaError_t e = cudaMemsetAsync(Y, 0, sizeof(float) * (size_t)batch * (size_t)rows, stream);
+    if (e != cudaSuccess) return (int)e;
+    const int nt = batch > 8 ? 2 : 1;
+    MmaParams p{};
+    size_t x_bytes = 0, stage_bytes = 0;
+    if (!mma_plan(fmt, cols, nt, p.chunk_cols, p.ring, x_bytes, stage_bytes)) return (int)cudaErrorInvalidValue;
+    p.W = static_cast<const uint8_t*>(W);
+    p.X = X;
+    p.Y = Y;
+    p.fault = fault;
+    p.rows = rows;
+    p.cols = cols;
+    p.row_bytes = (int64_t)lw_row_bytes(fmt, cols);
+    p.batch = batch;
+    p.x_off = kMmaHeader;
+    p.w_off = (uint32_t)((kMmaHeader + x_bytes + 127) / 128 * 128);
+    const size_t smem_bytes = p.w_off + (size_t)p.ring * stage_bytes;
+    const int64_t n_stages = (cols / kStageCols) * ((rows + kStageRows - 1) / kStageRows);
+    int grid = mma_sm_count();
+    if ((int64_t)grid > n_stages) grid = (int)n_stages;
+    alignas(64) CUtensorMap wmap;
+    if (!make_weight_map(&wmap, W, rows, p.row_bytes, (int)(stage_bytes / kStageRows))) return (int)cudaErrorInvalidValue;
+    if (fmt == LW_Q4_0)
+        return nt == 1 ? launch_mma<MmaQ40, 1>(p, wmap, grid, smem_bytes, stream)
+                       : launch_mma<MmaQ40, 2>(p, wmap, grid, smem_bytes, stream);
+    return nt == 1 ? launch_mma<MmaQ80, 1>(p, wmap, grid, smem_bytes, stream)
+                   : launch_mma<MmaQ80, 2>(p, wmap, grid, smem_bytes, stream);
+}
+
+}  // namespace lw

@@ -18,7 +18,7 @@ FORMATS = {"f16": F16, "q8_0": Q8_0, "q4_0": Q4_0, "q4_K": Q4_K, "q6_K": Q6_K, "
 BITS_PER_WEIGHT = {F16: 16.0, Q8_0: 8.5, Q4_0: 4.5, Q4_K: 4.5, Q6_K: 6.5625, Q5_K: 5.5, Q2_K: 2.625, Q4_1: 5.0,
                    Q5_0: 5.5, Q5_1: 6.0}
 
-VARIANT_AUTO, VARIANT_GENERIC, VARIANT_STREAM, VARIANT_IDOT, VARIANT_TILE = 0, 1, 2, 3, 4
+VARIANT_AUTO, VARIANT_GENERIC, VARIANT_STREAM, VARIANT_IDOT, VARIANT_TILE, VARIANT_MMA = 0, 1, 2, 3, 4, 5
 
 OK = 0
 ERR_FORMAT, ERR_SHAPE, ERR_NULL, ERR_ALIGN, ERR_BATCH, ERR_NONFINITE, ERR_CUDA, ERR_DEVICE = (

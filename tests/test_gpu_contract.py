@@ -20,7 +20,8 @@ pytestmark = pytest.mark.gpu
 FMTS = [lw.F16, lw.Q8_0, lw.Q4_0, lw.Q4_K, lw.Q6_K, lw.Q5_K, lw.Q2_K, lw.Q4_1, lw.Q5_0, lw.Q5_1]
 ALL_VARIANTS = [lw.VARIANT_AUTO, lw.VARIANT_GENERIC, lw.VARIANT_STREAM, lw.VARIANT_IDOT]
 # the extra term E = c * sum_k What_k * A_k of the header's accuracy statement, per launched variant
-C_EXTRA = {lw.VARIANT_GENERIC: 0.0, lw.VARIANT_STREAM: 2.0 ** -16, lw.VARIANT_IDOT: 2.0 ** -18}
+C_EXTRA = {lw.VARIANT_GENERIC: 0.0, lw.VARIANT_STREAM: 2.0 ** -16, lw.VARIANT_IDOT: 2.0 ** -18, lw.VARIANT_TILE: 0.0,
+           lw.VARIANT_MMA: 0.0}
 
 
 @pytest.fixture(autouse=True)
@@ -93,10 +94,13 @@ def test_outliers_on_zero_weights_stay_inside_the_stated_bound(fmt, variant, zer
     assert worst <= 1.0, "variant %d launched %d: error / bound = %.3g" % (variant, launched, worst)
 
 
+@pytest.mark.parametrize("kernel", [lw.VARIANT_TILE, lw.VARIANT_MMA])
 @pytest.mark.parametrize("fmt", [lw.Q8_0, lw.Q4_0])
-def test_tile_kernel_needs_no_extra_term(fmt):
-    # the batched tile kernel decodes every weight exactly before it multiplies: the plain tolerance holds on
-    # the same adversarial activations (eight columns, each with its own outliers), as the header states
+def test_batched_kernels_need_no_extra_term(fmt, kernel):
+    # the batched fp32 tile kernel decodes every weight exactly before it multiplies, and the tensor-core kernel
+    # multiplies exact integer codes with three bf16 terms that add up to the activation exactly: the plain
+    # tolerance holds on the same adversarial activations (eight columns, each with its own outliers), as the
+    # header states
     rows, cols, batch = 48, 4096, 8
     cols_x = []
     for b in range(batch):
@@ -104,15 +108,27 @@ def test_tile_kernel_needs_no_extra_term(fmt):
         cols_x.append(np.roll(X[0], 0) * (1.0 + b))
     X = np.stack(cols_x).astype(np.float32)
     y_ref, s_ref = oracle.matvec(fmt, blocks, rows, cols, X, batch)
-    lw.set_variant(lw.VARIANT_TILE)
-    assert lw.query_variant(fmt, rows, cols, batch) == lw.VARIANT_TILE
-    y = _run(fmt, blocks, rows, cols, X, lw.VARIANT_TILE, batch)
+    lw.set_variant(kernel)
+    assert lw.query_variant(fmt, rows, cols, batch) == kernel
+    y = _run(fmt, blocks, rows, cols, X, kernel, batch)
     worst = float((np.abs(y.astype(np.float64) - y_ref) / (RTOL * s_ref + ATOL)).max())
-    assert worst <= 1.0, "tile kernel: error / tolerance = %.3g" % worst
+    assert worst <= 1.0, "kernel %d: error / tolerance = %.3g" % (kernel, worst)
     # and a non-finite activation reaches every output of its column only
-    X[3, 100] = np.nan
-    y = _run(fmt, blocks, rows, cols, X, lw.VARIANT_TILE, batch)
-    assert not np.isfinite(y[3]).any() and np.isfinite(np.delete(y, 3, axis=0)).all()
+    for bad in (np.nan, np.inf, -np.inf):
+        Xb = X.copy()
+        Xb[3, 100] = bad
+        y = _run(fmt, blocks, rows, cols, Xb, kernel, batch)
+        assert not np.isfinite(y[3]).any() and np.isfinite(np.delete(y, 3, axis=0)).all()
+    # extreme magnitudes survive the three-term split: a huge value (the sums of code * x stay finite up to about
+    # 2^115, the limit the header states for the batched kernels) and a denormal
+    Xe = np.zeros((batch, cols), np.float32)
+    Xe[0, 7] = 1e30
+    Xe[1, 9] = 1e-41
+    Xe[2, :] = 2.0 ** -100
+    y_ref, s_ref = oracle.matvec(fmt, blocks, rows, cols, Xe, batch)
+    y = _run(fmt, blocks, rows, cols, Xe, kernel, batch)
+    finite = np.isfinite(y_ref.astype(np.float32))
+    assert (np.abs(y.astype(np.float64) - y_ref)[finite] <= (RTOL * s_ref + ATOL)[finite]).all()
 
 
 @pytest.mark.parametrize("variant", ALL_VARIANTS)

@@ -67,11 +67,9 @@ def test_matvec_batched(variant, fmt, batch):
 @pytest.mark.parametrize("rows,cols", [(1, 1024), (63, 2048), (64, 1024), (65, 4096), (333, 3072), (1000, 14336),
                                        (70000, 1024)])
 def test_matvec_tile_kernel(fmt, batch, rows, cols):
-    # the batched fp32 tile kernel (AUTO's choice for q8_0 / q4_0 when cols is a multiple of 1024): ragged row
+    # the batched fp32 tile kernel (on request; q8_0 / q4_0 when cols is a multiple of 1024): ragged row
     # counts around its 64-row stages, one to fourteen column chunks, passes of 4 and 8 columns, several CTAs
-    # per SM (70000 rows); forced and automatic selection must agree
-    lw.set_variant(lw.VARIANT_AUTO)
-    assert lw.query_variant(fmt, rows, cols, batch) == (lw.VARIANT_TILE if batch >= 7 else lw.VARIANT_IDOT)
+    # per SM (70000 rows)
     lw.set_variant(lw.VARIANT_TILE)
     assert lw.query_variant(fmt, rows, cols, batch) == lw.VARIANT_TILE
     blocks = quantized_weights(fmt, rows, cols, seed=59, tensor_id=fmt, outlier_p=0.01)
@@ -79,7 +77,24 @@ def test_matvec_tile_kernel(fmt, batch, rows, cols):
     y_ref, s_ref = oracle.matvec(fmt, blocks, rows, cols, X, batch, nthreads=8)
     y = gpu_matvec(fmt, blocks, rows, cols, X, batch, lw.VARIANT_TILE)
     check_matvec(y, y_ref, s_ref, "tile fmt %d %dx%d batch %d" % (fmt, rows, cols, batch))
-    y = gpu_matvec(fmt, blocks, rows, cols, X, batch, lw.VARIANT_AUTO)      # tile passes + a column-wise remainder
+
+
+@pytest.mark.parametrize("fmt", [lw.Q8_0, lw.Q4_0])
+@pytest.mark.parametrize("batch", [2, 3, 7, 8, 9, 16])
+@pytest.mark.parametrize("rows,cols", [(1, 256), (15, 512), (16, 1024), (17, 768), (255, 2048), (256, 1024), (257, 4096),
+                                       (333, 3072), (1000, 14336), (4096, 1280), (70000, 1024)])
+def test_matvec_mma_kernel(fmt, batch, rows, cols):
+    # the batched tensor-core kernel (AUTO's choice for q8_0 / q4_0 from three columns on when cols is a multiple of
+    # 256): ragged row counts around its 16-row fragments and 256-row stages, chunks of 256 / 512 / 1024 columns,
+    # one and two groups of eight columns, more stages than CTAs (70000 rows) and fewer (1 row)
+    lw.set_variant(lw.VARIANT_AUTO)
+    assert lw.query_variant(fmt, rows, cols, batch) == (lw.VARIANT_MMA if batch >= 3 else lw.VARIANT_IDOT)
+    blocks = quantized_weights(fmt, rows, cols, seed=61, tensor_id=fmt, outlier_p=0.01)
+    X = synth.activations(61, batch, batch, cols)
+    y_ref, s_ref = oracle.matvec(fmt, blocks, rows, cols, X, batch, nthreads=8)
+    y = gpu_matvec(fmt, blocks, rows, cols, X, batch, lw.VARIANT_MMA)
+    check_matvec(y, y_ref, s_ref, "mma fmt %d %dx%d batch %d" % (fmt, rows, cols, batch))
+    y = gpu_matvec(fmt, blocks, rows, cols, X, batch, lw.VARIANT_AUTO)
     check_matvec(y, y_ref, s_ref, "auto fmt %d %dx%d batch %d" % (fmt, rows, cols, batch))
 
 

@@ -131,10 +131,19 @@ def test_variant_controls():
     assert lw.query_variant(lw.Q4_K, 4096, 4096, 1) == lw.VARIANT_IDOT
     assert lw.query_variant(lw.F16, 4096, 4096, 1) == lw.VARIANT_STREAM
     assert lw.query_variant(lw.Q4_K, 4096, 4096, 2) == lw.VARIANT_IDOT       # one integer-dot pass per column
-    assert lw.query_variant(lw.Q4_0, 4096, 4096, 16) == lw.VARIANT_TILE      # fp32 tile kernel: q8_0 / q4_0, cols % 1024 == 0
-    assert lw.query_variant(lw.Q8_0, 128256, 4096, 7) == lw.VARIANT_TILE
-    assert lw.query_variant(lw.Q8_0, 128256, 4096, 6) == lw.VARIANT_IDOT        # fewer than 7 columns: one pass per column
-    assert lw.query_variant(lw.Q4_0, 4096, 4096 + 512, 16) == lw.VARIANT_IDOT  # cols not a multiple of 1024: one pass per column
+    assert lw.query_variant(lw.Q4_0, 4096, 4096, 16) == lw.VARIANT_MMA       # tensor-core kernel: q8_0 / q4_0, cols % 256 == 0
+    assert lw.query_variant(lw.Q8_0, 128256, 4096, 3) == lw.VARIANT_MMA
+    assert lw.query_variant(lw.Q8_0, 128256, 4096, 2) == lw.VARIANT_IDOT        # two columns: one pass per column
+    assert lw.query_variant(lw.Q4_0, 4096, 4096 + 512, 16) == lw.VARIANT_MMA
+    assert lw.query_variant(lw.Q4_0, 4096, 4096 + 128, 16) == lw.VARIANT_GENERIC  # cols % 256 != 0: no streaming kernel
+    lw.set_variant(lw.VARIANT_TILE)
+    assert lw.query_variant(lw.Q4_0, 4096, 4096, 16) == lw.VARIANT_TILE      # fp32 tile kernel on request, cols % 1024 == 0
+    assert lw.query_variant(lw.Q4_0, 4096, 4096 + 512, 16) != lw.VARIANT_TILE
+    lw.set_variant(lw.VARIANT_MMA)
+    assert lw.query_variant(lw.Q4_0, 4096, 4096, 2) == lw.VARIANT_MMA
+    assert lw.query_variant(lw.Q4_K, 4096, 4096, 8) != lw.VARIANT_MMA
+    assert lw.query_variant(lw.Q4_0, 4096, 4096, 1) == lw.VARIANT_IDOT        # batch 1: falls back
+    lw.set_variant(lw.VARIANT_AUTO)
     assert lw.query_variant(lw.Q4_1, 4096, 4096, 16) == lw.VARIANT_IDOT
     assert lw.query_variant(lw.Q8_0, 16, 96, 3) == lw.VARIANT_GENERIC       # cols % 256 != 0: tiled fp32 kernel
     assert lw.query_variant(lw.Q6_K, 4096, 4096, 1) == lw.VARIANT_IDOT
