@@ -54,6 +54,9 @@ def arithmetic_of(fmt, batch):
         return "f32 in/out; f16 weights widened, fp32 FMA"
     if batch == 1:
         return "f32 in/out; activations as 24-bit block fixed point, int32 dp4a sums, fp32 block scales"
+    if fmt in ("q8_0", "q4_0") and batch >= 3:
+        return ("f32 in/out; exact bf16 weight codes x three-term bf16 split of the fp32 activations on the tensor cores "
+                "(mma m16n8k16), fp32 accumulation and block scales")
     return "f32 in/out; batch > 1: per-column passes of the batch-1 kernel (24-bit block fixed point, int32 dp4a) or fp32 FMA tiles"
 
 
@@ -300,7 +303,9 @@ def run_step(args):
     X = X_host.cuda()
     Y = torch.zeros(yt, dtype=torch.float32, device="cuda")
 
-    lw.set_overlap(not args.no_overlap)
+    # batch > 1: the weights are model parameters that nothing on the stream writes, so the tensor-core kernel may
+    # start streaming them while the previous kernel finishes (overlap level 2)
+    lw.set_overlap(0 if args.no_overlap else (2 if batch > 1 else 1))
     if args.tuning_table:
         log("tuning table: %d entries" % lw.load_tuning_table(args.tuning_table))
     wptr, xptr, yptr = W.data_ptr(), X.data_ptr(), Y.data_ptr()
@@ -437,6 +442,15 @@ def run_step(args):
             others[mode] = describe(mode, timer.time(replays[mode], args.steps, 3))
     if batch == 1 and "per-call" not in to_time and not args.only and not args.no_graph:
         others["per-call"] = describe("per-call", timer.time(capture(torch, enqueue_per_call), args.steps, 3))
+    if batch > 1 and all(lw.query_variant(fmt_id, r, c, batch) == lw.VARIANT_MMA for _, r, c in shapes):
+        # the same step with the tensor-core kernel switched off: the fp32 tile kernel where it applies (passes of 8
+        # and 4 columns), else what the heuristics would pick without it
+        lw.set_variant(lw.VARIANT_TILE)
+        kinds = {lw.query_variant(fmt_id, r, c, batch) for _, r, c in shapes}
+        d = describe("per-call", timer.time(capture(torch, enqueue_per_call, not args.no_graph), args.steps, 3))
+        d["issue"] = "per-call, tensor cores off (LW_VARIANT_TILE forced; variants launched: %s)" % sorted(kinds)
+        others["fp32_only"] = d
+        lw.set_variant(lw.VARIANT_AUTO)
 
     # ---- end to end through the host-buffer entry points of the C ABI, pinned host memory on both sides, the
     # copies inside the timed region.  Batch 1: ONE lw_matvec_sequence_host call per step (the step's activation
@@ -526,7 +540,25 @@ def run_step(args):
             int(TRAFFIC_RATIO[args.workload] * (wbytes + abytes) / launches_per_step)
             if args.workload in TRAFFIC_RATIO and batch == 1 else None, ceiling),
     }
-    if batch > 1:
+    mma_served = batch > 1 and all(lw.query_variant(fmt_id, r, c, batch) == lw.VARIANT_MMA for _, r, c in shapes)
+    if mma_served:
+        # the tensor-core kernel: every weight-column product is issued three times (one per bf16 term of the
+        # activation), in groups of eight columns; state the tensor work against the measured bf16 GEMM peak
+        cols8 = 8 * ((batch + 7) // 8)
+        issued = sum(2.0 * r * c * cols8 * 3 for _, r, c in shapes)
+        try:
+            with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as fh:
+                tpeak, tsrc = float(json.load(fh)["bf16_tflops_sustained"]), "measured (MEASURED_PEAKS.json bf16_tflops_sustained)"
+        except Exception:
+            tpeak, tsrc = 1400.0, "fallback (1.4 PFLOP/s sustained, earlier measurement on this pool)"
+        result["roofline_tensor"] = {
+            "bound": "tensor", "achieved": round(issued / (step_ms * 1e-3) / 1e12, 1), "peak": tpeak, "peak_source": tsrc,
+            "unit": "TFLOP/s", "frac": round(issued / (step_ms * 1e-3) / 1e12 / tpeak, 4),
+            "what": "bf16 products issued (3 terms x columns rounded up to 8) over the step time; the peak is the tcgen05 "
+                    "GEMM figure, which the warp-level mma used here cannot reach (measured: one m16n8k16 per ~10 cycles "
+                    "per SM sub-partition, i.e. about 470 TFLOP/s for the whole GPU); the HBM roofline in `roofline` is the "
+                    "bound a faster contraction would hit first"}
+    elif batch > 1:
         # the binding bound from batch 2 on is instruction issue, not HBM: state it with its derivation
         flops = sum(2.0 * r * c * batch for _, r, c in shapes)
         alu_peak = 148 * 128 * 1.965e9 * 2 / 1e12

@@ -274,7 +274,10 @@ int lw_plan_info(int fmt, int64_t rows, int64_t cols, int* out6);
  * launches carry the programmatic-serialisation attribute, so a mat-vec kernel's CTAs may be placed and
  * run their set-up (barrier initialisation, launch latency) while the previous kernel on the stream is
  * still finishing; they wait for that kernel to complete before they request any of W or X or write Y.
- * Default off.  Process-wide. */
+ * enabled = 2: the same, and the batched tensor-core kernel (LW_VARIANT_MMA) may start streaming W before
+ * the previous kernel has completed -- only for weights that no work still pending on the stream writes
+ * (model parameters); X and Y are still not touched before.  Other values: LW_ERR_FORMAT.
+ * Default off (0).  Process-wide. */
 int lw_set_overlap(int enabled);
 
 /* Decode attention of ONE query token over a block-quantised KV cache [Sec 3.2 "FlashAttention": the

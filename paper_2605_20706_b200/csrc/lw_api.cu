@@ -159,7 +159,7 @@ int lw_matvec(int fmt, const void* W_blocks, int64_t rows, int64_t cols, const f
     int err;
     const int variant = pick_variant(fmt, rows, cols, batch);
     if (variant == LW_VARIANT_MMA) {
-        err = launch_matvec_mma(fmt, W_blocks, rows, cols, X, Y, batch, s);
+        err = launch_matvec_mma(fmt, W_blocks, rows, cols, X, Y, batch, g_overlap.load(), s);
     } else if (variant == LW_VARIANT_TILE && forced_variant() == LW_VARIANT_AUTO) {
         // passes of seven or eight columns through the tile kernel, the remainder through the batch-1 kernel
         const int tiled = batch - (batch % 8 >= kTileMinColumns ? 0 : batch % 8);
@@ -400,7 +400,8 @@ int lw_debug_drop_copy(int unit) {
 }
 
 int lw_set_overlap(int enabled) {
-    g_overlap.store(enabled ? 1 : 0);
+    if (enabled < 0 || enabled > 2) return LW_ERR_FORMAT;
+    g_overlap.store(enabled);
     return LW_OK;
 }
 

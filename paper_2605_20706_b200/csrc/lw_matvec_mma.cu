@@ -68,6 +68,7 @@ struct MmaParams {
     int batch;            // columns of this launch (<= 8 NT)
     int chunk_cols;       // 256, 512 or 1024: columns whose activations are resident at a time
     int ring;             // stages in the ring (2..kMaxRing)
+    int early_weights;    // the weight copies may start before the previous kernel on the stream has completed
     uint32_t x_off, w_off;
 };
 
@@ -230,6 +231,17 @@ __device__ __forceinline__ void split3(float x, uint32_t& h1, uint32_t& h2, uint
     h3 = __float_as_uint(r2) >> 16;                     // at most eight significant bits are left: exact
 }
 
+// Clears Y for the kernel below.  Launched like it (see launch_matvec_mma): lets its successor start its set-up
+// at once and waits for its predecessor before it writes.
+__global__ void __launch_bounds__(256) zero_kernel(float4* __restrict__ y, int64_t quads, float* __restrict__ tail,
+                                                   int n_tail) {
+    grid_launch_dependents();
+    grid_dependency_wait();
+    const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < quads; i += (int64_t)gridDim.x * blockDim.x) y[i] = z;
+    if (blockIdx.x == 0 && (int)threadIdx.x < n_tail) tail[threadIdx.x] = 0.f;
+}
+
 // Where a CTA is in its range of stages: chunk c, row stage rs, sub-stage j of the chunk, ring slot and the
 // parity of the slot's current use.  Stepped without divisions.
 struct Cursor {
@@ -280,6 +292,11 @@ __global__ void __launch_bounds__(kMmaThreads, 1) matvec_mma_kernel(const __grid
     const int64_t first = n_stages * blockIdx.x / gridDim.x, last = n_stages * (blockIdx.x + 1) / gridDim.x;
     const int ring = p.ring;
 
+    // With programmatic dependent launch this kernel may have been placed while its predecessor on the stream
+    // (the kernel that clears Y, and through it everything before) is still running: its successor may be placed
+    // from now on, and nothing of X or Y is touched before grid_dependency_wait() returns.  Both are no-ops in
+    // an ordinary launch.
+    grid_launch_dependents();
     if (tid == 0) {
         for (int s = 0; s < kMaxRing; ++s) {
             mbar_init(&full[s], 1);
@@ -293,6 +310,7 @@ __global__ void __launch_bounds__(kMmaThreads, 1) matvec_mma_kernel(const __grid
     if (warp == kMmaWarps) {
         // ------------------------------------------------------------- producer (one thread) ---
         if (lane != 0) return;
+        if (!p.early_weights) grid_dependency_wait();
         const uint64_t policy = l2_evict_first_policy();
         const int count = (int)(last - first);
         Cursor cur;
@@ -320,6 +338,7 @@ __global__ void __launch_bounds__(kMmaThreads, 1) matvec_mma_kernel(const __grid
     }
 
     // ------------------------------------------------------------------- compute warps ---
+    grid_dependency_wait();
     const int g = lane >> 2, t = lane & 3;
     const uint32_t xs = smem_u32(smem + p.x_off);
     // this lane's B fragments: column g of each group of eight, slots 8 t .. 8 t + 7 of a block of 32
@@ -436,7 +455,8 @@ __global__ void __launch_bounds__(kMmaThreads, 1) matvec_mma_kernel(const __grid
 }
 
 template <class T, int NT>
-int launch_mma(const MmaParams& p, const CUtensorMap& wmap, int grid, size_t smem_bytes, cudaStream_t stream) {
+int launch_mma(const MmaParams& p, const CUtensorMap& wmap, int grid, size_t smem_bytes, bool overlap,
+               cudaStream_t stream) {
     static bool attr_set[64] = {false};
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
@@ -446,8 +466,17 @@ int launch_mma(const MmaParams& p, const CUtensorMap& wmap, int grid, size_t sme
         if (e != cudaSuccess) return (int)e;
         if (dev >= 0 && dev < 64) attr_set[dev] = true;
     }
-    matvec_mma_kernel<T, NT><<<(unsigned)grid, kMmaThreads, smem_bytes, stream>>>(p, wmap);
-    return (int)cudaGetLastError();
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(kMmaThreads);
+    cfg.dynamicSmemBytes = smem_bytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = overlap ? 1 : 0;
+    return (int)cudaLaunchKernelEx(&cfg, matvec_mma_kernel<T, NT>, p, wmap);
 }
 
 // cuTensorMapEncodeTiled through the runtime's driver entry point lookup (no link against the driver library)
@@ -514,13 +543,31 @@ bool matvec_mma_supported(int fmt, int64_t rows, int64_t cols, int batch) {
 }
 
 // Arguments are validated by the caller; returns a cudaError_t as int.
+// overlap: 0 ordinary launches; 1 programmatic dependent launch (set-up overlaps the previous kernel's end);
+// 2 the same, and the weight copies start before the previous kernel has completed.
 int launch_matvec_mma(int fmt, const void* W, int64_t rows, int64_t cols, const float* X, float* Y, int batch,
-                      cudaStream_t stream) {
+                      int overlap, cudaStream_t stream) {
     int* fault = device_fault_word();
     if (!fault) return (int)cudaErrorInvalidValue;
-    // the kernel adds every (chunk, row stage) share into Y
-    cudaError_t e = cudaMemsetAsync(Y, 0, sizeof(float) * (size_t)batch * (size_t)rows, stream);
-    if (e != cudaSuccess) return (int)e;
+    // the kernel adds every (chunk, row stage) share into Y: clear it first (Y is 16-byte aligned)
+    {
+        const int64_t n = (int64_t)batch * rows, quads = n / 4;
+        int64_t blocks = (quads + 255) / 256;
+        if (blocks < 1) blocks = 1;
+        if (blocks > 4 * mma_sm_count()) blocks = 4 * mma_sm_count();
+        cudaLaunchConfig_t cfg{};
+        cfg.gridDim = dim3((unsigned)blocks);
+        cfg.blockDim = dim3(256);
+        cfg.stream = stream;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr;
+        cfg.numAttrs = overlap ? 1 : 0;
+        const cudaError_t e = cudaLaunchKernelEx(&cfg, zero_kernel, reinterpret_cast<float4*>(Y), quads, Y + 4 * quads,
+                                                 (int)(n - 4 * quads));
+        if (e != cudaSuccess) return (int)e;
+    }
     const int nt = batch > 8 ? 2 : 1;
     MmaParams p{};
     size_t x_bytes = 0, stage_bytes = 0;
@@ -533,6 +580,7 @@ int launch_matvec_mma(int fmt, const void* W, int64_t rows, int64_t cols, const 
     p.cols = cols;
     p.row_bytes = (int64_t)lw_row_bytes(fmt, cols);
     p.batch = batch;
+    p.early_weights = overlap >= 2;
     p.x_off = kMmaHeader;
     p.w_off = (uint32_t)((kMmaHeader + x_bytes + 127) / 128 * 128);
     const size_t smem_bytes = p.w_off + (size_t)p.ring * stage_bytes;
@@ -542,10 +590,10 @@ int launch_matvec_mma(int fmt, const void* W, int64_t rows, int64_t cols, const 
     alignas(64) CUtensorMap wmap;
     if (!make_weight_map(&wmap, W, rows, p.row_bytes, (int)(stage_bytes / kStageRows))) return (int)cudaErrorInvalidValue;
     if (fmt == LW_Q4_0)
-        return nt == 1 ? launch_mma<MmaQ40, 1>(p, wmap, grid, smem_bytes, stream)
-                       : launch_mma<MmaQ40, 2>(p, wmap, grid, smem_bytes, stream);
-    return nt == 1 ? launch_mma<MmaQ80, 1>(p, wmap, grid, smem_bytes, stream)
-                   : launch_mma<MmaQ80, 2>(p, wmap, grid, smem_bytes, stream);
+        return nt == 1 ? launch_mma<MmaQ40, 1>(p, wmap, grid, smem_bytes, overlap != 0, stream)
+                       : launch_mma<MmaQ40, 2>(p, wmap, grid, smem_bytes, overlap != 0, stream);
+    return nt == 1 ? launch_mma<MmaQ80, 1>(p, wmap, grid, smem_bytes, overlap != 0, stream)
+                   : launch_mma<MmaQ80, 2>(p, wmap, grid, smem_bytes, overlap != 0, stream);
 }
 
 }  // namespace lw

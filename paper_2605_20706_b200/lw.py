@@ -270,8 +270,9 @@ def query_variant(fmt: int, rows: int, cols: int, batch: int = 1) -> int:
     return rc
 
 
-def set_overlap(enabled: bool) -> None:
-    _check(lib().lw_set_overlap(1 if enabled else 0), "lw_set_overlap")
+def set_overlap(enabled) -> None:
+    """False / 0: ordinary launches; True / 1: programmatic dependent launch; 2: and early weight streaming."""
+    _check(lib().lw_set_overlap(int(enabled)), "lw_set_overlap")
 
 
 def set_tuning(worker_groups: int = 0, stages: int = 0, stage_kb: int = 0) -> None:
