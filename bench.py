@@ -380,6 +380,13 @@ def run_step(args):
         lw.set_sequence_mode(lw.SEQ_PERSISTENT)
         lw.matvec_sequence(fmt_id, seq_arr, seq_ws, stream=stream)
 
+    def enqueue_grouped(stream):
+        # batch > 1: one lw_matvec_group_batch call per group (q/k/v together, gate/up together, the rest alone)
+        for g in groups:
+            c = shapes[g[0]][2]
+            lw.matvec_group(fmt_id, c, [(wptr + offs[j], shapes[j][1], xptr + 4 * xoffs[g[0]], yptr + 4 * yoffs[j])
+                                        for j in g], stream, batch=batch)
+
     modes = {"launches": (enqueue_launches, len(groups),
                           "one lw_matvec_sequence call per step, run as one grouped launch per phase (q/k/v together, "
                           "gate/up together, the rest alone: %d launches per step) chained with programmatic dependent "
@@ -388,9 +395,12 @@ def run_step(args):
                             "one lw_matvec_sequence call per step, run as ONE persistent kernel (grid-wide barrier before "
                             "each dependent mat-vec, weight ring kept filling across boundaries): 1 launch per step"),
              "per-call": (enqueue_per_call, ncalls, "one lw_matvec call per mat-vec (%d launches per step), q/k/v and "
-                                                    "gate/up on parallel graph branches" % ncalls)}
+                                                    "gate/up on parallel graph branches" % ncalls),
+             "grouped": (enqueue_grouped, len(groups),
+                         "one lw_matvec_group_batch call per group of mat-vecs that share their activations (q/k/v together, "
+                         "gate/up together, the rest alone: %d calls per step)" % len(groups))}
     if batch > 1:
-        to_time = ["per-call"]
+        to_time = ["per-call", "grouped"] if args.issue == "auto" else [args.issue]
     elif args.issue == "auto":
         to_time = ["launches", "persistent"]
     else:
@@ -408,6 +418,10 @@ def run_step(args):
     headline = min(to_time, key=lambda m: timings[m])
     one_step = replays[headline]
     launches_per_step = modes[headline][1]
+    if batch > 1 and all(lw.query_variant(fmt_id, r, c, batch) == lw.VARIANT_MMA for _, r, c in shapes):
+        # the tensor-core kernel adds into Y: with overlap every mat-vec's Y is cleared by a small kernel of its own in
+        # front (chained by programmatic dependent launch); without, the main kernel clears it itself
+        launches_per_step += 0 if args.no_overlap else ncalls
 
     # ---- device-resident timing of the headline mode, clocks sampled during it
     for _ in range(max(3, args.warmup)):
@@ -1186,8 +1200,8 @@ def main():
     ap.add_argument("--layers", type=int, default=None, help="use fewer layers (debugging only)")
     ap.add_argument("--only", default=None, help="comma-separated substrings: keep only matching mat-vecs "
                                                   "(profiling of single kernels)")
-    ap.add_argument("--issue", default="auto", choices=["auto", "launches", "persistent", "per-call"],
-                    help="how the step's mat-vecs are issued at batch 1 (auto: time launches and persistent, report the faster)")
+    ap.add_argument("--issue", default="auto", choices=["auto", "launches", "persistent", "per-call", "grouped"],
+                    help="how the step is issued (auto: batch 1 times launches and persistent, batch > 1 per-call and grouped; the faster is the headline)")
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--serial", action="store_true", help="per-call mode on one branch: every mat-vec waits for the previous one")
     ap.add_argument("--no-overlap", action="store_true")

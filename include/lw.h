@@ -156,6 +156,14 @@ typedef struct {
 } lw_group_item;
 int lw_matvec_group(int fmt, int64_t cols, int n_items, const lw_group_item* items, void* stream);
 
+/* The same with `batch` activation columns per item (1..16): X of an item is batch * cols floats, Y batch * rows
+ * floats, laid out as in lw_matvec.  batch 1 is lw_matvec_group.  From two columns on, q8_0 / q4_0 with cols a
+ * multiple of 256 run all items in ONE launch of the tensor-core kernel (LW_VARIANT_MMA, unless another variant
+ * is forced; items that follow one another and share their X pointer share its converted copy); everything else
+ * is run item by item with lw_matvec.  Errors as lw_matvec (LW_ERR_BATCH for batch outside 1..16); a call that
+ * fails validation enqueues nothing. */
+int lw_matvec_group_batch(int fmt, int64_t cols, int n_items, const lw_group_item* items, int batch, void* stream);
+
 /* A whole chain of batch-1 mat-vecs of one format in ONE call [Sec 3.1, 3.2: the runtime groups operations
  * into compute passes; the whole mat-vec chain of a decode step is one pass here].  The items run in the
  * order given.  Consecutive items that read the same X (same pointer, same cols) and are not flagged

@@ -25,6 +25,18 @@ static int forced_variant() {
     return g_variant.load();
 }
 
+// Does the current device take cooperative launches (kernels whose CTAs wait for one another)?
+static bool cooperative_launch_ok() {
+    static int coop[64] = {0};          // 0 unknown, 1 yes, -1 no
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return false;
+    if (coop[dev] == 0) {
+        int v = 0;
+        coop[dev] = (cudaDeviceGetAttribute(&v, cudaDevAttrCooperativeLaunch, dev) == cudaSuccess && v) ? 1 : -1;
+    }
+    return coop[dev] == 1;
+}
+
 static bool misaligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
 
 static int check_matvec_args(int fmt, const void* W, int64_t rows, int64_t cols, const void* X,
@@ -159,7 +171,10 @@ int lw_matvec(int fmt, const void* W_blocks, int64_t rows, int64_t cols, const f
     int err;
     const int variant = pick_variant(fmt, rows, cols, batch);
     if (variant == LW_VARIANT_MMA) {
-        err = launch_matvec_mma(fmt, W_blocks, rows, cols, X, Y, batch, g_overlap.load(), s);
+        // without overlap: one cooperative launch that clears Y itself; with it: a clearing kernel and the main
+        // kernel chained by programmatic dependent launch
+        const int ov = g_overlap.load();
+        err = launch_matvec_mma(fmt, W_blocks, rows, cols, X, Y, batch, ov, ov == 0 && cooperative_launch_ok(), s);
     } else if (variant == LW_VARIANT_TILE && forced_variant() == LW_VARIANT_AUTO) {
         // passes of seven or eight columns through the tile kernel, the remainder through the batch-1 kernel
         const int tiled = batch - (batch % 8 >= kTileMinColumns ? 0 : batch % 8);
@@ -198,6 +213,37 @@ int lw_matvec(int fmt, const void* W_blocks, int64_t rows, int64_t cols, const f
     else
         err = launch_matvec_generic(fmt, W_blocks, rows, cols, X, Y, batch, s);
     return err == 0 ? LW_OK : LW_ERR_CUDA;
+}
+
+int lw_matvec_group_batch(int fmt, int64_t cols, int n_items, const lw_group_item* items, int batch, void* stream) {
+    if (batch == 1) return lw_matvec_group(fmt, cols, n_items, items, stream);
+    if (lw_block_elems(fmt) == 0) return LW_ERR_FORMAT;
+    if (!items) return LW_ERR_NULL;
+    if (n_items < 1 || n_items > 8) return LW_ERR_SHAPE;
+    const void* W[8];
+    const float* X[8];
+    float* Y[8];
+    int64_t rows[8];
+    for (int j = 0; j < n_items; ++j) {
+        const int rc = check_matvec_args(fmt, items[j].W_blocks, items[j].rows, cols, items[j].X, items[j].Y, batch);
+        if (rc != LW_OK) return rc;
+        W[j] = items[j].W_blocks;
+        X[j] = items[j].X;
+        Y[j] = items[j].Y;
+        rows[j] = items[j].rows;
+    }
+    const int forced = forced_variant();
+    if ((forced == LW_VARIANT_AUTO || forced == LW_VARIANT_MMA) && matvec_mma_group_supported(fmt, cols, n_items, rows, batch)) {
+        const int ov = g_overlap.load();
+        const int err = launch_matvec_mma_group(fmt, cols, n_items, W, rows, X, Y, batch, ov,
+                                                ov == 0 && cooperative_launch_ok(), static_cast<cudaStream_t>(stream));
+        return err == 0 ? LW_OK : LW_ERR_CUDA;
+    }
+    for (int j = 0; j < n_items; ++j) {
+        const int rc = lw_matvec(fmt, W[j], rows[j], cols, X[j], Y[j], batch, stream);
+        if (rc != LW_OK) return rc;
+    }
+    return LW_OK;
 }
 
 int lw_matvec_group(int fmt, int64_t cols, int n_items, const lw_group_item* items, void* stream) {
@@ -248,14 +294,7 @@ int lw_matvec_sequence(int fmt, int n_items, const lw_seq_item* items, void* wor
         if (rc != LW_OK) return rc;
         if (items[j].flags & ~LW_SEQ_DEPENDENT) return LW_ERR_FORMAT;
     }
-    static int coop[64] = {0};          // 0 unknown, 1 yes, -1 no
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return LW_ERR_CUDA;
-    if (dev >= 0 && dev < 64 && coop[dev] == 0) {
-        int v = 0;
-        coop[dev] = (cudaDeviceGetAttribute(&v, cudaDevAttrCooperativeLaunch, dev) == cudaSuccess && v) ? 1 : -1;
-    }
-    const bool can = dev >= 0 && dev < 64 && coop[dev] == 1;
+    const bool can = cooperative_launch_ok();
     const bool streaming = forced_variant() == LW_VARIANT_AUTO && matvec_sequence_supported(fmt, n_items, items);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (streaming && can && g_sequence_mode.load() == LW_SEQ_PERSISTENT) {

@@ -52,7 +52,12 @@ int launch_matvec_tile(int fmt, const void* W, int64_t rows, int64_t cols, const
 // accumulation): q8_0 and q4_0 with cols a multiple of 256.  The launch clears Y first (the kernel adds into it).
 bool matvec_mma_supported(int fmt, int64_t rows, int64_t cols, int batch);
 int launch_matvec_mma(int fmt, const void* W, int64_t rows, int64_t cols, const float* X, float* Y, int batch,
-                      int overlap, cudaStream_t stream);
+                      int overlap, bool self_clear, cudaStream_t stream);
+// The same for up to eight matrices of one format and width in one launch (each with its own X and Y).
+bool matvec_mma_group_supported(int fmt, int64_t cols, int n_items, const int64_t* rows, int batch);
+int launch_matvec_mma_group(int fmt, int64_t cols, int n_items, const void* const* W, const int64_t* rows,
+                            const float* const* X, float* const* Y, int batch, int overlap, bool self_clear,
+                            cudaStream_t stream);
 // Tunables of the streaming kernels (0 = automatic) and the geometry they lead to for a shape.
 void set_stream_tuning(int worker_groups, int stages, int stage_kb);
 // Per-shape tunables (all zero erases the entry); make_plan uses them where the process-wide ones are 0.

@@ -48,7 +48,13 @@
 namespace lw {
 namespace {
 
-constexpr int kMmaWarps = 16;                         // compute warps
+#ifndef LW_MMA_WARPS
+#define LW_MMA_WARPS 16
+#endif
+constexpr int kMmaWarps = LW_MMA_WARPS;               // compute warps
+constexpr int kCtasPerSm = 16 / kMmaWarps;
+constexpr int kSmemPerCta = kCtasPerSm == 1 ? 227 * 1024 : 113 * 1024;
+constexpr int kXR = 8 * 64 / (32 * kMmaWarps);        // quads per thread, piece and group of eight columns
 constexpr int kMmaComputeThreads = 32 * kMmaWarps;
 constexpr int kMmaThreads = kMmaComputeThreads + 32;  // plus the producer warp
 constexpr int kStageRows = 16 * kMmaWarps;            // 256
@@ -57,18 +63,42 @@ constexpr int kStageUnits = kStageCols / 64;
 constexpr int kMaxRing = 4;
 constexpr int kXPad = 64;                             // bytes after each column of a plane: 16-byte loads of lanes
                                                       // (g, t) at 64 g + 16 t cover 128 distinct bytes per quarter warp
-constexpr int kMmaHeader = 128;                       // barriers and the stop flag
+constexpr int kMmaHeader = 128;                       // barriers, the stop flag and the grid barrier's generation
+constexpr uint32_t kGridPolls = 1u << 20;             // polls of the generation word (~0.5 us each) before giving up
 
-struct MmaParams {
-    const uint8_t* W;
+// Grid barrier of the self-clearing launches: {count, generation}.  A launch holds every SM (one CTA per SM,
+// cooperative), so two launches never use it at the same time; the last CTA to arrive resets the count and
+// bumps the generation, which leaves the words ready for the next launch whatever happened in this one.
+__device__ unsigned g_mma_grid_barrier[2] = {0u, 0u};
+
+constexpr int kMmaMaxItems = 8;                       // matrices of one width per launch
+
+// One matrix of a launch: its row stages are numbered rs_begin .. rs_begin + ceil(rows / 256) - 1 in the launch.
+struct MmaItem {
     const float* X;
     float* Y;
+    int64_t rows;
+    int rs_begin;
+    int same_x_end;       // first row stage (of the launch) after the run of matrices that share this X
+};
+
+struct MmaMaps {
+    CUtensorMap m[kMmaMaxItems];
+};
+
+struct MmaParams {
     int* fault;
-    int64_t rows, cols, row_bytes;
+    int64_t cols;
+    MmaItem item[kMmaMaxItems];
+    int n_items;
+    int total_rs;         // row stages of all matrices
     int batch;            // columns of this launch (<= 8 NT)
     int chunk_cols;       // 256, 512 or 1024: columns whose activations are resident at a time
     int ring;             // stages in the ring (2..kMaxRing)
     int early_weights;    // the weight copies may start before the previous kernel on the stream has completed
+    int self_clear;       // cooperative launch: the CTAs clear Y themselves and meet at a grid barrier before the
+                          // first sum is added (no clearing kernel in front)
+    unsigned* grid_bar;   // {arrival count, generation} of that barrier, owned by the library
     uint32_t x_off, w_off;
 };
 
@@ -242,37 +272,43 @@ __global__ void __launch_bounds__(256) zero_kernel(float4* __restrict__ y, int64
     if (blockIdx.x == 0 && (int)threadIdx.x < n_tail) tail[threadIdx.x] = 0.f;
 }
 
-// Where a CTA is in its range of stages: chunk c, row stage rs, sub-stage j of the chunk, ring slot and the
-// parity of the slot's current use.  Stepped without divisions.
+// Where a CTA is in its range of stages: chunk c, row stage rs (numbered through all matrices of the launch) of
+// matrix `it`, sub-stage j of the chunk, ring slot and the parity of the slot's current use.  Stepped without
+// divisions.
 struct Cursor {
-    int c, rs, j, slot;
+    int c, rs, j, slot, it;
     uint32_t parity;
-    __device__ __forceinline__ void init(int64_t first, int spc, int n_rs) {
+    __device__ __forceinline__ void init(const MmaParams& p, int64_t first, int spc) {
         const int64_t pair = first / spc;
         j = (int)(first - pair * spc);
-        c = (int)(pair / n_rs);
-        rs = (int)(pair - (int64_t)c * n_rs);
+        c = (int)(pair / p.total_rs);
+        rs = (int)(pair - (int64_t)c * p.total_rs);
+        it = 0;
+        while (it + 1 < p.n_items && rs >= p.item[it + 1].rs_begin) ++it;
         slot = 0;
         parity = 0;
     }
-    __device__ __forceinline__ void step(int spc, int n_rs, int ring) {
+    __device__ __forceinline__ void step(const MmaParams& p, int spc, int ring) {
         if (++slot == ring) {
             slot = 0;
             parity ^= 1u;
         }
         if (++j == spc) {
             j = 0;
-            if (++rs == n_rs) {
+            if (++rs == p.total_rs) {
                 rs = 0;
+                it = 0;
                 ++c;
+            } else if (it + 1 < p.n_items && rs >= p.item[it + 1].rs_begin) {
+                ++it;
             }
         }
     }
 };
 
 template <class T, int NT>
-__global__ void __launch_bounds__(kMmaThreads, 1) matvec_mma_kernel(const __grid_constant__ MmaParams p,
-                                                                    const __grid_constant__ CUtensorMap wmap) {
+__global__ void __launch_bounds__(kMmaThreads, kCtasPerSm) matvec_mma_kernel(const __grid_constant__ MmaParams p,
+                                                                             const __grid_constant__ MmaMaps maps) {
     extern __shared__ __align__(128) uint8_t smem[];
     uint64_t* full = reinterpret_cast<uint64_t*>(smem);               // [kMaxRing]
     uint64_t* empty = full + kMaxRing;                                // [kMaxRing]
@@ -286,7 +322,7 @@ __global__ void __launch_bounds__(kMmaThreads, 1) matvec_mma_kernel(const __grid
     const uint32_t x_pitch = 2u * Kx + kXPad;                         // bytes between columns of a plane
     const uint32_t plane_pitch = NB * x_pitch;
     const int spc = Kx / kStageCols;                                  // stages per (chunk, row stage)
-    const int n_rs = (int)((p.rows + kStageRows - 1) / kStageRows);
+    const int n_rs = p.total_rs;
     const int n_chunks = (int)(p.cols / Kx);
     const int64_t n_stages = (int64_t)n_chunks * n_rs * spc;
     const int64_t first = n_stages * blockIdx.x / gridDim.x, last = n_stages * (blockIdx.x + 1) / gridDim.x;
@@ -306,6 +342,7 @@ __global__ void __launch_bounds__(kMmaThreads, 1) matvec_mma_kernel(const __grid
         fence_barrier_init();
     }
     __syncthreads();
+    volatile unsigned* gen_seen = reinterpret_cast<volatile unsigned*>(smem + 72);   // generation before this CTA arrived
 
     if (warp == kMmaWarps) {
         // ------------------------------------------------------------- producer (one thread) ---
@@ -314,9 +351,9 @@ __global__ void __launch_bounds__(kMmaThreads, 1) matvec_mma_kernel(const __grid
         const uint64_t policy = l2_evict_first_policy();
         const int count = (int)(last - first);
         Cursor cur;
-        cur.init(first, spc, n_rs);
+        cur.init(p, first, spc);
         int n = 0;
-        for (; n < count; ++n, cur.step(spc, n_rs, ring)) {
+        for (; n < count; ++n, cur.step(p, spc, ring)) {
             if (*stop) break;
             if (n >= ring && !mbar_wait_bounded(&empty[cur.slot], cur.parity ^ 1u)) {   // the slot's previous use
                 atomicExch(p.fault, (int)FAULT_BULK_WAIT_TIMEOUT);
@@ -324,8 +361,9 @@ __global__ void __launch_bounds__(kMmaThreads, 1) matvec_mma_kernel(const __grid
                 break;
             }
             mbar_expect_tx(&full[cur.slot], kStageBytes);   // a box always delivers all its bytes (zeros past the end)
-            tensor_load_2d(smem + p.w_off + (size_t)cur.slot * kStageBytes, &wmap, (cur.c * spc + cur.j) * (kPiece / 4),
-                           cur.rs * kStageRows, &full[cur.slot], policy);
+            tensor_load_2d(smem + p.w_off + (size_t)cur.slot * kStageBytes, &maps.m[cur.it],
+                           (cur.c * spc + cur.j) * (kPiece / 4), (cur.rs - p.item[cur.it].rs_begin) * kStageRows,
+                           &full[cur.slot], policy);
         }
         if (*stop) {
             // the consumers have stopped waiting: make sure nothing is still landing in shared memory (stage m,
@@ -339,6 +377,31 @@ __global__ void __launch_bounds__(kMmaThreads, 1) matvec_mma_kernel(const __grid
 
     // ------------------------------------------------------------------- compute warps ---
     grid_dependency_wait();
+    if (p.self_clear) {
+        // this CTA's share of Y, then its arrival at the grid barrier; nobody adds into Y before the barrier
+        // has completed (checked before the first flush, by which time it normally has)
+        for (int it = 0; it < p.n_items; ++it) {
+            const int64_t n = (int64_t)p.batch * p.item[it].rows, quads = n / 4;
+            const int64_t q0 = quads * blockIdx.x / gridDim.x, q1 = quads * (blockIdx.x + 1) / gridDim.x;
+            float4* y4 = reinterpret_cast<float4*>(p.item[it].Y);
+            for (int64_t i = q0 + tid; i < q1; i += kMmaComputeThreads) y4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (blockIdx.x == 0 && tid < (int)(n - 4 * quads)) p.item[it].Y[4 * quads + tid] = 0.f;
+        }
+        compute_barrier();
+        if (tid == 0) {
+            unsigned gen, prev;
+            asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(gen) : "l"(p.grid_bar + 1) : "memory");
+            *gen_seen = gen;
+            // release: the stores above (ordered before this thread by the barrier) become visible device-wide to
+            // whoever observes the new generation; acquire: the last CTA to arrive has seen everybody's
+            asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(prev) : "l"(p.grid_bar) : "memory");
+            if (prev == gridDim.x - 1) {
+                asm volatile("st.relaxed.gpu.global.u32 [%0], %1;" ::"l"(p.grid_bar), "r"(0u) : "memory");
+                asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(p.grid_bar + 1) : "memory");
+            }
+        }
+    }
+    bool cleared = !p.self_clear;       // may this warp add into Y yet?
     const int g = lane >> 2, t = lane & 3;
     const uint32_t xs = smem_u32(smem + p.x_off);
     // this lane's B fragments: column g of each group of eight, slots 8 t .. 8 t + 7 of a block of 32
@@ -350,54 +413,75 @@ __global__ void __launch_bounds__(kMmaThreads, 1) matvec_mma_kernel(const __grid
     for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
         for (int i = 0; i < 4; ++i) y[nt][i] = 0.f;
-    int cur_c = -1, cur_rs = -1;
+    int cur_c = -1, cur_rs = -1, cur_it = 0;
+    const float* cur_x = nullptr;
 
     auto flush = [&]() {
         // add this warp's sums of (chunk, row stage cur_rs) into Y: rows g and g + 8 of the warp's 16, columns
         // 8 nt + 2 t and 8 nt + 2 t + 1
-        const int64_t r = (int64_t)cur_rs * kStageRows + 16 * warp + g;
+        if (!cleared) {
+            // the grid barrier: every CTA has cleared its share of Y once the generation has moved on
+            if (lane == 0 && !*stop) {
+                const unsigned gen0 = *gen_seen;       // written before the barriers of the first conversion
+                unsigned gen = gen0;
+                for (uint32_t i = 0; i < kGridPolls && gen == gen0; ++i)
+                    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(gen) : "l"(p.grid_bar + 1) : "memory");
+                if (gen == gen0) {
+                    atomicExch(p.fault, (int)FAULT_GRID_BARRIER_TIMEOUT);
+                    *stop = 1;
+                }
+            }
+            __syncwarp();
+            cleared = true;
+        }
+        const MmaItem& m = p.item[cur_it];
+        const int64_t r = (int64_t)(cur_rs - m.rs_begin) * kStageRows + 16 * warp + g;
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
                 const int b = 8 * nt + 2 * t + (i & 1);
                 const int64_t rr = r + (i >> 1) * 8;
-                if (b < p.batch && rr < p.rows) atomicAdd(p.Y + (int64_t)b * p.rows + rr, y[nt][i]);
+                if (b < p.batch && rr < m.rows) atomicAdd(m.Y + (int64_t)b * m.rows + rr, y[nt][i]);
                 y[nt][i] = 0.f;
             }
     };
 
     const int count = (int)(last - first);
     Cursor cur;
-    cur.init(first, spc, n_rs);
-    for (int n = 0; n < count; ++n, cur.step(spc, n_rs, ring)) {
+    cur.init(p, first, spc);
+    for (int n = 0; n < count; ++n, cur.step(p, spc, ring)) {
         const int c = cur.c, rs = cur.rs, j = cur.j, slot = cur.slot;
+        const MmaItem& mat = p.item[cur.it];
         if (c != cur_c || rs != cur_rs) {
             if (cur_rs >= 0) flush();
             cur_rs = rs;
+            cur_it = cur.it;
         }
-        if (c != cur_c) {
+        if (c != cur_c || mat.X != cur_x) {
             // the chunk's activations as three bf16 planes: plane s, column b.  Inside a block of 32 the order is
             // the one the fragments want: slots 8 q .. 8 q + 3 hold k = 4 q .. 4 q + 3 and slots 8 q + 4 .. 8 q + 7
             // hold k = 16 + 4 q .., so a lane reads both halves of its B operand with one 16-byte load.
             cur_c = c;
+            cur_x = mat.X;
             compute_barrier();                          // every warp is done with the previous chunk
             // Only the 256-column pieces this CTA's stages inside the chunk will read (all of them once it has
             // `spc` or more stages here); a piece is 64 quads of each column: one quad per thread and group of
             // eight columns.  All loads are issued before the first conversion.
-            const int64_t in_chunk = (int64_t)(n_rs - rs) * spc - j;
+            const int64_t in_chunk = (int64_t)(mat.same_x_end - rs) * spc - j;    // stages ahead that read this X
             const int left = count - n;
             const int m = (int)(in_chunk < left ? in_chunk : left);
-            float4 v[4][NT];
+            float4 v[4][NT * kXR];
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
                 const int jj = (j + q) % spc;
 #pragma unroll
-                for (int nt = 0; nt < NT; ++nt) {
-                    const int b = 8 * nt + (tid >> 6), k4 = jj * (kStageCols / 4) + (tid & 63);
+                for (int nt = 0; nt < NT * kXR; ++nt) {
+                    const int idx = tid + nt * kMmaComputeThreads;
+                    const int b = idx >> 6, k4 = jj * (kStageCols / 4) + (idx & 63);
                     v[q][nt] = make_float4(0.f, 0.f, 0.f, 0.f);
                     if (q < spc && q < m && b < p.batch)
-                        v[q][nt] = __ldg(reinterpret_cast<const float4*>(p.X + (int64_t)b * p.cols + (int64_t)c * Kx) + k4);
+                        v[q][nt] = __ldg(reinterpret_cast<const float4*>(mat.X + (int64_t)b * p.cols + (int64_t)c * Kx) + k4);
                 }
             }
 #pragma unroll
@@ -405,8 +489,9 @@ __global__ void __launch_bounds__(kMmaThreads, 1) matvec_mma_kernel(const __grid
                 const int jj = (j + q) % spc;
                 if (q < spc && q < m) {
 #pragma unroll
-                    for (int nt = 0; nt < NT; ++nt) {
-                        const int b = 8 * nt + (tid >> 6), k4 = jj * (kStageCols / 4) + (tid & 63);
+                    for (int nt = 0; nt < NT * kXR; ++nt) {
+                        const int idx = tid + nt * kMmaComputeThreads;
+                        const int b = idx >> 6, k4 = jj * (kStageCols / 4) + (idx & 63);
                         uint32_t h[3][4];
                         split3(v[q][nt].x, h[0][0], h[1][0], h[2][0]);
                         split3(v[q][nt].y, h[0][1], h[1][1], h[2][1]);
@@ -430,8 +515,8 @@ __global__ void __launch_bounds__(kMmaThreads, 1) matvec_mma_kernel(const __grid
                 *stop = 1;
             }
         }
-        const int64_t r0 = (int64_t)rs * kStageRows;
-        if (r0 + 16 * warp < p.rows) {
+        const int64_t r0 = (int64_t)(rs - mat.rs_begin) * kStageRows;
+        if (r0 + 16 * warp < mat.rows) {
             const uint32_t row = wrow + (uint32_t)slot * kStageBytes, wt = row + 4u * t;
             uint32_t xp[NT][3];
 #pragma unroll
@@ -455,14 +540,15 @@ __global__ void __launch_bounds__(kMmaThreads, 1) matvec_mma_kernel(const __grid
 }
 
 template <class T, int NT>
-int launch_mma(const MmaParams& p, const CUtensorMap& wmap, int grid, size_t smem_bytes, bool overlap,
+int launch_mma(const MmaParams& p, const MmaMaps& maps, int grid, size_t smem_bytes, bool overlap,
                cudaStream_t stream) {
+    // self-clearing launches are cooperative (their CTAs wait for one another) and ordinary in stream order
     static bool attr_set[64] = {false};
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return (int)e;
     if (dev < 0 || dev >= 64 || !attr_set[dev]) {
-        e = cudaFuncSetAttribute(matvec_mma_kernel<T, NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+        e = cudaFuncSetAttribute(matvec_mma_kernel<T, NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemPerCta);
         if (e != cudaSuccess) return (int)e;
         if (dev >= 0 && dev < 64) attr_set[dev] = true;
     }
@@ -472,11 +558,16 @@ int launch_mma(const MmaParams& p, const CUtensorMap& wmap, int grid, size_t sme
     cfg.dynamicSmemBytes = smem_bytes;
     cfg.stream = stream;
     cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    if (p.self_clear) {
+        attr[0].id = cudaLaunchAttributeCooperative;
+        attr[0].val.cooperative = 1;
+    } else {
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+    }
     cfg.attrs = attr;
-    cfg.numAttrs = overlap ? 1 : 0;
-    return (int)cudaLaunchKernelEx(&cfg, matvec_mma_kernel<T, NT>, p, wmap);
+    cfg.numAttrs = (p.self_clear || overlap) ? 1 : 0;
+    return (int)cudaLaunchKernelEx(&cfg, matvec_mma_kernel<T, NT>, p, maps);
 }
 
 // cuTensorMapEncodeTiled through the runtime's driver entry point lookup (no link against the driver library)
@@ -520,7 +611,7 @@ int mma_sm_count() {
 bool mma_plan(int fmt, int64_t cols, int nt, int& chunk_cols, int& ring, size_t& x_bytes, size_t& stage_bytes) {
     const int block_bytes = fmt == LW_Q4_0 ? 18 : 34;
     stage_bytes = (size_t)kStageRows * (kStageCols / 32) * block_bytes;
-    const size_t budget = 227 * 1024 - kMmaHeader;
+    const size_t budget = kSmemPerCta - kMmaHeader;
     for (int kx = 1024; kx >= 256; kx /= 2) {
         if (cols % kx != 0) continue;
         x_bytes = (size_t)3 * 8 * nt * (2 * kx + kXPad);
@@ -542,16 +633,33 @@ bool matvec_mma_supported(int fmt, int64_t rows, int64_t cols, int batch) {
     return rows >= 1 && rows <= (int64_t)1 << 30;
 }
 
-// Arguments are validated by the caller; returns a cudaError_t as int.
+bool matvec_mma_group_supported(int fmt, int64_t cols, int n_items, const int64_t* rows, int batch) {
+    if (n_items < 1 || n_items > kMmaMaxItems) return false;
+    int64_t total_rs = 0;
+    for (int i = 0; i < n_items; ++i) {
+        if (!matvec_mma_supported(fmt, rows[i], cols, batch)) return false;
+        total_rs += (rows[i] + kStageRows - 1) / kStageRows;
+    }
+    return total_rs * (cols / kStageCols) < ((int64_t)1 << 31);
+}
+
+// Up to kMmaMaxItems matrices of one format and width in one launch, each with its own X and Y (matrices that
+// share an X pointer and follow one another share its converted copy).  Arguments are validated by the caller;
+// returns a cudaError_t as int.
 // overlap: 0 ordinary launches; 1 programmatic dependent launch (set-up overlaps the previous kernel's end);
-// 2 the same, and the weight copies start before the previous kernel has completed.
-int launch_matvec_mma(int fmt, const void* W, int64_t rows, int64_t cols, const float* X, float* Y, int batch,
-                      int overlap, cudaStream_t stream) {
+// 2 the same, and the weight copies start before the previous kernel has completed.  self_clear: one cooperative
+// launch whose CTAs clear Y themselves (no clearing kernel, no programmatic launch).
+int launch_matvec_mma_group(int fmt, int64_t cols, int n_items, const void* const* W, const int64_t* rows,
+                            const float* const* X, float* const* Y, int batch, int overlap, bool self_clear,
+                            cudaStream_t stream) {
     int* fault = device_fault_word();
     if (!fault) return (int)cudaErrorInvalidValue;
+    unsigned* grid_bar = nullptr;
+    if (self_clear && cudaGetSymbolAddress(reinterpret_cast<void**>(&grid_bar), g_mma_grid_barrier) != cudaSuccess)
+        return (int)cudaErrorInvalidValue;
     // the kernel adds every (chunk, row stage) share into Y: clear it first (Y is 16-byte aligned)
-    {
-        const int64_t n = (int64_t)batch * rows, quads = n / 4;
+    for (int i = 0; i < n_items && !self_clear; ++i) {
+        const int64_t n = (int64_t)batch * rows[i], quads = n / 4;
         int64_t blocks = (quads + 255) / 256;
         if (blocks < 1) blocks = 1;
         if (blocks > 4 * mma_sm_count()) blocks = 4 * mma_sm_count();
@@ -564,36 +672,53 @@ int launch_matvec_mma(int fmt, const void* W, int64_t rows, int64_t cols, const 
         attr[0].val.programmaticStreamSerializationAllowed = 1;
         cfg.attrs = attr;
         cfg.numAttrs = overlap ? 1 : 0;
-        const cudaError_t e = cudaLaunchKernelEx(&cfg, zero_kernel, reinterpret_cast<float4*>(Y), quads, Y + 4 * quads,
-                                                 (int)(n - 4 * quads));
+        const cudaError_t e = cudaLaunchKernelEx(&cfg, zero_kernel, reinterpret_cast<float4*>(Y[i]), quads,
+                                                 Y[i] + 4 * quads, (int)(n - 4 * quads));
         if (e != cudaSuccess) return (int)e;
     }
     const int nt = batch > 8 ? 2 : 1;
     MmaParams p{};
     size_t x_bytes = 0, stage_bytes = 0;
     if (!mma_plan(fmt, cols, nt, p.chunk_cols, p.ring, x_bytes, stage_bytes)) return (int)cudaErrorInvalidValue;
-    p.W = static_cast<const uint8_t*>(W);
-    p.X = X;
-    p.Y = Y;
+    alignas(64) MmaMaps maps;
+    const int64_t row_bytes = (int64_t)lw_row_bytes(fmt, cols);
+    int rs = 0;
+    for (int i = 0; i < n_items; ++i) {
+        p.item[i].X = X[i];
+        p.item[i].Y = Y[i];
+        p.item[i].rows = rows[i];
+        p.item[i].rs_begin = rs;
+        rs += (int)((rows[i] + kStageRows - 1) / kStageRows);
+        if (!make_weight_map(&maps.m[i], W[i], rows[i], row_bytes, (int)(stage_bytes / kStageRows)))
+            return (int)cudaErrorInvalidValue;
+    }
+    for (int i = n_items - 1; i >= 0; --i)          // end of the run of matrices that read the same X
+        p.item[i].same_x_end = (i + 1 < n_items && X[i + 1] == X[i]) ? p.item[i + 1].same_x_end : (i + 1 < n_items ? p.item[i + 1].rs_begin : rs);
+    for (int i = n_items; i < kMmaMaxItems; ++i) maps.m[i] = maps.m[0];
+    p.n_items = n_items;
+    p.total_rs = rs;
     p.fault = fault;
-    p.rows = rows;
     p.cols = cols;
-    p.row_bytes = (int64_t)lw_row_bytes(fmt, cols);
     p.batch = batch;
-    p.early_weights = overlap >= 2;
+    p.early_weights = overlap >= 2 && !self_clear;
+    p.self_clear = self_clear ? 1 : 0;
+    p.grid_bar = grid_bar;
     p.x_off = kMmaHeader;
     p.w_off = (uint32_t)((kMmaHeader + x_bytes + 127) / 128 * 128);
     const size_t smem_bytes = p.w_off + (size_t)p.ring * stage_bytes;
-    const int64_t n_stages = (cols / kStageCols) * ((rows + kStageRows - 1) / kStageRows);
-    int grid = mma_sm_count();
-    if ((int64_t)grid > n_stages) grid = (int)n_stages;
-    alignas(64) CUtensorMap wmap;
-    if (!make_weight_map(&wmap, W, rows, p.row_bytes, (int)(stage_bytes / kStageRows))) return (int)cudaErrorInvalidValue;
+    const int64_t n_stages = (cols / kStageCols) * (int64_t)rs;
+    int grid = kCtasPerSm * mma_sm_count();
+    if ((int64_t)grid > n_stages && !self_clear) grid = (int)n_stages;   // self-clearing: every SM, so launches never overlap
     if (fmt == LW_Q4_0)
-        return nt == 1 ? launch_mma<MmaQ40, 1>(p, wmap, grid, smem_bytes, overlap != 0, stream)
-                       : launch_mma<MmaQ40, 2>(p, wmap, grid, smem_bytes, overlap != 0, stream);
-    return nt == 1 ? launch_mma<MmaQ80, 1>(p, wmap, grid, smem_bytes, overlap != 0, stream)
-                   : launch_mma<MmaQ80, 2>(p, wmap, grid, smem_bytes, overlap != 0, stream);
+        return nt == 1 ? launch_mma<MmaQ40, 1>(p, maps, grid, smem_bytes, overlap != 0, stream)
+                       : launch_mma<MmaQ40, 2>(p, maps, grid, smem_bytes, overlap != 0, stream);
+    return nt == 1 ? launch_mma<MmaQ80, 1>(p, maps, grid, smem_bytes, overlap != 0, stream)
+                   : launch_mma<MmaQ80, 2>(p, maps, grid, smem_bytes, overlap != 0, stream);
+}
+
+int launch_matvec_mma(int fmt, const void* W, int64_t rows, int64_t cols, const float* X, float* Y, int batch,
+                      int overlap, bool self_clear, cudaStream_t stream) {
+    return launch_matvec_mma_group(fmt, cols, 1, &W, &rows, &X, &Y, batch, overlap, self_clear, stream);
 }
 
 }  // namespace lw

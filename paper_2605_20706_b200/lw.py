@@ -28,7 +28,7 @@ ERR_WORKSPACE = -9
 LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "liblw.so")
 
 EXPORTS = ("lw_block_elems", "lw_block_bytes", "lw_row_bytes", "lw_status_string", "lw_quantize",
-           "lw_dequant", "lw_matvec", "lw_matvec_group", "lw_matvec_host", "lw_set_variant", "lw_query_variant",
+           "lw_dequant", "lw_matvec", "lw_matvec_group", "lw_matvec_group_batch", "lw_matvec_host", "lw_set_variant", "lw_query_variant",
            "lw_set_overlap", "lw_device_status", "lw_set_tuning", "lw_plan_info", "lw_attn_decode",
            "lw_attn_workspace_bytes", "lw_attn_decode_static", "lw_set_attn_variant", "lw_query_attn_variant",
            "lw_debug_drop_copy", "lw_matvec_sequence", "lw_matvec_sequence_workspace_bytes", "lw_probe_read", "lw_set_sequence_mode", "lw_matvec_sequence_host", "lw_set_shape_tuning", "lw_clear_shape_tuning")
@@ -61,6 +61,8 @@ def lib() -> ctypes.CDLL:
     L.lw_matvec.restype, L.lw_matvec.argtypes = c_int, [c_int, vp, i64, i64, vp, vp, c_int, vp]
     L.lw_matvec_group.restype = c_int
     L.lw_matvec_group.argtypes = [c_int, i64, c_int, vp, vp]
+    L.lw_matvec_group_batch.restype = c_int
+    L.lw_matvec_group_batch.argtypes = [c_int, i64, c_int, vp, c_int, vp]
     L.lw_matvec_host.restype = c_int
     L.lw_matvec_host.argtypes = [c_int, vp, i64, i64, vp, vp, vp, vp, c_int, vp]
     L.lw_set_variant.restype, L.lw_set_variant.argtypes = c_int, [c_int]
@@ -157,13 +159,17 @@ class GroupItem(ctypes.Structure):
                 ("Y", ctypes.c_void_p)]
 
 
-def matvec_group(fmt: int, cols: int, items, stream=None) -> None:
-    """items: sequence of (W_blocks, rows, X, Y); one launch for all of them (batch 1)."""
+def matvec_group(fmt: int, cols: int, items, stream=None, batch: int = 1) -> None:
+    """items: sequence of (W_blocks, rows, X, Y); one launch for all of them where the kernels allow it."""
     arr = (GroupItem * len(items))()
     for j, (w, rows, x, y) in enumerate(items):
         arr[j].W_blocks, arr[j].rows, arr[j].X, arr[j].Y = _addr(w) or None, rows, _addr(x) or None, _addr(y) or None
-    _check(lib().lw_matvec_group(fmt, cols, len(items), ctypes.cast(arr, ctypes.c_void_p),
-                                 _stream_handle(stream)), "lw_matvec_group")
+    if batch == 1:
+        _check(lib().lw_matvec_group(fmt, cols, len(items), ctypes.cast(arr, ctypes.c_void_p),
+                                     _stream_handle(stream)), "lw_matvec_group")
+    else:
+        _check(lib().lw_matvec_group_batch(fmt, cols, len(items), ctypes.cast(arr, ctypes.c_void_p), batch,
+                                           _stream_handle(stream)), "lw_matvec_group_batch")
 
 
 class SeqItem(ctypes.Structure):

@@ -98,6 +98,38 @@ def test_matvec_mma_kernel(fmt, batch, rows, cols):
     check_matvec(y, y_ref, s_ref, "auto fmt %d %dx%d batch %d" % (fmt, rows, cols, batch))
 
 
+@pytest.mark.parametrize("overlap", [0, 1, 2])
+@pytest.mark.parametrize("fmt", [lw.Q8_0, lw.Q4_0])
+def test_matvec_mma_launch_modes(fmt, overlap):
+    # the two ways the tensor-core kernel gets a cleared Y: one cooperative launch whose CTAs clear it and meet at a
+    # grid barrier (no overlap), or a clearing kernel chained to it by programmatic dependent launch (overlap 1;
+    # 2: weights requested before the previous kernel has completed).  A chain of calls into ping-pong buffers,
+    # so a call's Y is the X the call before last read, replayed several times.
+    batch, dims = 5, [1024, 768, 2048, 1024, 512]
+    mats = [quantized_weights(fmt, dims[j + 1], dims[j], seed=63 + j, tensor_id=fmt) for j in range(len(dims) - 1)]
+    wd = [torch.from_numpy(m).cuda() for m in mats]
+    x0 = synth.activations(63, 0, batch, dims[0])
+    bufs = [torch.zeros(batch * max(dims), dtype=torch.float32, device="cuda") for _ in range(2)]
+    lw.set_variant(lw.VARIANT_MMA)
+    lw.set_overlap(overlap)
+    try:
+        for _ in range(3):
+            bufs[0][:x0.size] = torch.from_numpy(x0.reshape(-1)).cuda()
+            for j in range(len(mats)):
+                lw.matvec(fmt, wd[j], dims[j + 1], dims[j], bufs[j & 1], bufs[(j + 1) & 1], batch)
+            torch.cuda.synchronize()
+            assert lw.device_status() == 0
+            got = bufs[len(mats) & 1][:batch * dims[-1]].cpu().numpy().reshape(batch, dims[-1])
+            # the chain's rounding differences grow from layer to layer: compare the last layer against the oracle
+            # fed with the GPU's own input to that layer
+            x_in = bufs[(len(mats) - 1) & 1][:batch * dims[-2]].cpu().numpy().reshape(batch, dims[-2])
+            y_ref, s_ref = oracle.matvec(fmt, mats[-1], dims[-1], dims[-2], x_in, batch, nthreads=4)
+            check_matvec(got, y_ref, s_ref, "mma chain overlap %d" % overlap)
+    finally:
+        lw.set_overlap(0)
+        lw.set_variant(lw.VARIANT_AUTO)
+
+
 @pytest.mark.parametrize("variant", VARIANTS)
 def test_config1_q8_0_2048(variant):
     # the single q8_0 mat-vec of the first benchmark configuration: every output checked
@@ -260,6 +292,40 @@ def test_matvec_group(variant, fmt, cols, row_list):
         check_matvec(y.t.cpu().numpy(), y_ref, s_ref, "group item")
 
 
+@pytest.mark.parametrize("overlap", [0, 2])
+@pytest.mark.parametrize("batch", [2, 5, 12])
+@pytest.mark.parametrize("fmt", [lw.Q8_0, lw.Q4_0, lw.Q4_K])
+@pytest.mark.parametrize("cols,row_list,share", [(1024, [300, 77, 1000], True), (2048, [513, 256], True),
+                                                 (768, [40, 1, 255, 17, 256, 3, 700, 64], False), (4096, [37], True)])
+def test_matvec_group_batch(fmt, batch, overlap, cols, row_list, share):
+    # several matrices and several columns in one call: q8_0 / q4_0 go through one launch of the tensor-core kernel
+    # (shared or separate activations, ragged row counts around its 256-row stages, both launch modes), q4_K item by
+    # item through lw_matvec
+    lw.set_variant(lw.VARIANT_AUTO)
+    lw.set_overlap(overlap)
+    try:
+        x_shared = torch.from_numpy(synth.activations(64, 99, batch, cols)).cuda()
+        items, refs, keep = [], [], []
+        for j, rows in enumerate(row_list):
+            blocks = quantized_weights(fmt, rows, cols, seed=64 + j, tensor_id=fmt)
+            X = synth.activations(64, 99 if share else j, batch, cols)
+            w = torch.from_numpy(blocks).cuda()
+            x = x_shared if share else torch.from_numpy(X).cuda()
+            y = Guarded((batch, rows))
+            keep.append((w, x, y))
+            items.append((w, rows, x, y.t))
+            refs.append(oracle.matvec(fmt, blocks, rows, cols, X, batch, nthreads=4))
+        for _ in range(2):
+            lw.matvec_group(fmt, cols, items, batch=batch)
+        torch.cuda.synchronize()
+        assert lw.device_status() == 0
+        for (w, x, y), (y_ref, s_ref) in zip(keep, refs):
+            y.check("group item")
+            check_matvec(y.t.cpu().numpy(), y_ref, s_ref, "batched group item")
+    finally:
+        lw.set_overlap(0)
+
+
 def test_matvec_group_argument_errors():
     L = lw.lib()
     w = torch.zeros(4096, dtype=torch.uint8, device="cuda")
@@ -275,3 +341,10 @@ def test_matvec_group_argument_errors():
         lw.matvec_group(lw.Q8_0, 64, [(w, 4, None, y)])
     assert e.value.code == lw.ERR_NULL
     assert L.lw_matvec_group(lw.Q8_0, 64, 1, None, None) == lw.ERR_NULL
+    with pytest.raises(lw.LwError) as e:
+        lw.matvec_group(lw.Q8_0, 64, [(w, 4, x, y)], batch=17)
+    assert e.value.code == lw.ERR_BATCH
+    with pytest.raises(lw.LwError) as e:
+        lw.matvec_group(lw.Q8_0, 64, [(w, 4, x, y)] * 9, batch=4)
+    assert e.value.code == lw.ERR_SHAPE
+    assert L.lw_matvec_group_batch(lw.Q8_0, 64, 1, None, 4, None) == lw.ERR_NULL
