@@ -305,7 +305,8 @@ def run_step(args):
 
     # batch > 1: the weights are model parameters that nothing on the stream writes, so the tensor-core kernel may
     # start streaming them while the previous kernel finishes (overlap level 2)
-    lw.set_overlap(0 if args.no_overlap else (2 if batch > 1 else 1))
+    overlap_level = 0 if args.no_overlap else (args.overlap if args.overlap is not None else (2 if batch > 1 else 1))
+    lw.set_overlap(overlap_level)
     if args.tuning_table:
         log("tuning table: %d entries" % lw.load_tuning_table(args.tuning_table))
     wptr, xptr, yptr = W.data_ptr(), X.data_ptr(), Y.data_ptr()
@@ -418,10 +419,11 @@ def run_step(args):
     headline = min(to_time, key=lambda m: timings[m])
     one_step = replays[headline]
     launches_per_step = modes[headline][1]
-    if batch > 1 and all(lw.query_variant(fmt_id, r, c, batch) == lw.VARIANT_MMA for _, r, c in shapes):
+    mma_possible = batch > 1 and fmt in ("q8_0", "q4_0") and all(c % 256 == 0 for _, _, c in shapes)
+    if mma_possible and (headline == "grouped" or batch >= 3):
         # the tensor-core kernel adds into Y: with overlap every mat-vec's Y is cleared by a small kernel of its own in
         # front (chained by programmatic dependent launch); without, the main kernel clears it itself
-        launches_per_step += 0 if args.no_overlap else ncalls
+        launches_per_step += 0 if overlap_level == 0 else ncalls
 
     # ---- device-resident timing of the headline mode, clocks sampled during it
     for _ in range(max(3, args.warmup)):
@@ -1205,6 +1207,8 @@ def main():
     ap.add_argument("--no-graph", action="store_true")
     ap.add_argument("--serial", action="store_true", help="per-call mode on one branch: every mat-vec waits for the previous one")
     ap.add_argument("--no-overlap", action="store_true")
+    ap.add_argument("--overlap", type=int, default=None, choices=[0, 1, 2],
+                    help="lw_set_overlap level (default 1 at batch 1, 2 beyond: weights are parameters nothing on the stream writes)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=4.0)
     ap.add_argument("--ref-rows", type=int, default=512)
