@@ -48,13 +48,16 @@ SINGLE_WORKLOADS = ("q8_0_2048",)
 DEQUANT_WORKLOADS = tuple("dequant_" + f for f in FMT_ID)
 
 
+MMA_FORMATS = ("q8_0", "q4_0", "q4_K")       # formats the batched tensor-core kernel takes
+
+
 def arithmetic_of(fmt, batch):
     """What the kernels compute in (the `dtype` key): not a precision claim, the arithmetic that runs."""
     if fmt == "f16":
         return "f32 in/out; f16 weights widened, fp32 FMA"
     if batch == 1:
         return "f32 in/out; activations as 24-bit block fixed point, int32 dp4a sums, fp32 block scales"
-    if fmt in ("q8_0", "q4_0") and batch >= 3:
+    if fmt in MMA_FORMATS and batch >= 3:
         return ("f32 in/out; exact bf16 weight codes x three-term bf16 split of the fp32 activations on the tensor cores "
                 "(mma m16n8k16), fp32 accumulation and block scales")
     return "f32 in/out; batch > 1: per-column passes of the batch-1 kernel (24-bit block fixed point, int32 dp4a) or fp32 FMA tiles"
@@ -419,7 +422,7 @@ def run_step(args):
     headline = min(to_time, key=lambda m: timings[m])
     one_step = replays[headline]
     launches_per_step = modes[headline][1]
-    mma_possible = batch > 1 and fmt in ("q8_0", "q4_0") and all(c % 256 == 0 for _, _, c in shapes)
+    mma_possible = batch > 1 and fmt in MMA_FORMATS and all(c % 256 == 0 for _, _, c in shapes)
     if mma_possible and (headline == "grouped" or batch >= 3):
         # the tensor-core kernel adds into Y: with overlap every mat-vec's Y is cleared by a small kernel of its own in
         # front (chained by programmatic dependent launch); without, the main kernel clears it itself
@@ -514,7 +517,7 @@ def run_step(args):
     per_gpu_gbs = gbs / world
     kernel = ("matvec_seq_kernel" if headline == "persistent" else "matvec_stream_kernel") + \
         "<%s%s>" % ("Idot_" if fmt != "f16" else "", fmt)
-    if batch > 1 and fmt in ("q8_0", "q4_0") and (headline == "grouped" or batch >= 3) and all(c % 256 == 0 for _, _, c in shapes):
+    if batch > 1 and fmt in MMA_FORMATS and (headline == "grouped" or batch >= 3) and all(c % 256 == 0 for _, _, c in shapes):
         kernel = "matvec_mma_kernel<%s, %d>" % (fmt, 1 if batch <= 8 else 2)
     result = {
         "metric": METRIC,

@@ -1,4 +1,4 @@
-// Batched mat-vec on the tensor cores (batch 2..16, q4_0 and q8_0) [paper Sec 3.2: from a handful of columns on
+// Batched mat-vec on the tensor cores (batch 2..16; q4_0, q8_0 and q4_K) [paper Sec 3.2: from a handful of columns on
 // the mat-vec turns into a small mat-mat product, a dense contraction; Sec 3.3: one decode routine per format
 // spliced into a common skeleton].
 //
@@ -11,7 +11,8 @@
 //   * an fp32 activation is cut into three bf16 terms of eight significant bits each, by truncation:
 //     x = x1 + x2 + x3 exactly, so that code * x1 + code * x2 + code * x3, accumulated in fp32 by the tensor
 //     core, is the fp32-accumulated product with the exact activation.  A NaN or Inf stays one (in x1 or x2).
-// The accuracy is therefore that of the fp32 kernels: |y - y_ref| <= 1e-4 * sum|w x| + 1e-6 with no extra term.
+// The accuracy is therefore that of the fp32 kernels: |y - y_ref| <= 1e-4 * sum|w x| + 1e-6 with no extra term
+// (q4_0, q8_0; q4_K's sub-block offsets go onto fp32 sums of the activations and bring an extra term back, see MmaQ4K).
 //
 // Why mma.sync and not tcgen05.mma here: the A operand is the decoded weight, which exists only in registers
 // (18- and 34-byte blocks decode to fragments with byte permutes); tcgen05.mma reads A from shared or tensor
@@ -63,6 +64,7 @@ constexpr int kStageUnits = kStageCols / 64;
 constexpr int kMaxRing = 4;
 constexpr int kXPad = 64;                             // bytes after each column of a plane: 16-byte loads of lanes
                                                       // (g, t) at 64 g + 16 t cover 128 distinct bytes per quarter warp
+constexpr int kSxBlockBytes = 64;                     // block sums of the activations: [block of 32][16 columns] floats
 constexpr int kMmaHeader = 128;                       // barriers, the stop flag and the grid barrier's generation
 constexpr uint32_t kGridPolls = 1u << 20;             // polls of the generation word (~0.5 us each) before giving up
 
@@ -100,6 +102,7 @@ struct MmaParams {
                           // first sum is added (no clearing kernel in front)
     unsigned* grid_bar;   // {arrival count, generation} of that barrier, owned by the library
     uint32_t x_off, w_off;
+    uint32_t sx_off, tab_off;   // block sums of the activations and the warps' scale tables (formats that need them)
 };
 
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
@@ -125,6 +128,10 @@ __device__ __forceinline__ float lds_half(uint32_t base) {
     unsigned short h;
     asm volatile("ld.shared.u16 %0, [%1+%2];" : "=h"(h) : "r"(base), "n"(OFF));
     return __half2float(__ushort_as_half(h));
+}
+template <int OFF>
+__device__ __forceinline__ void lds_f32x2(uint32_t base, float& a, float& b) {
+    asm volatile("ld.shared.v2.f32 {%0, %1}, [%2+%3];" : "=f"(a), "=f"(b) : "r"(base), "n"(OFF));
 }
 template <int OFF>
 __device__ __forceinline__ void lds128(uint32_t base, uint32_t& a, uint32_t& b, uint32_t& c, uint32_t& d) {
@@ -171,9 +178,13 @@ __device__ __forceinline__ uint32_t bytes_to_bf16_128_plus(uint32_t v) {
 // p[2], p[3] = weights 16+4t .. 16+4t+3 (the k order the B fragments follow).  `wt` = shared-memory address of
 // the row's piece of the stage plus 4 t (t = lane % 4), OFF = byte offset of the two-block unit from there.
 struct MmaQ40 {
-    static constexpr int kBlockBytes = 18;
-    template <int OFF, int BLK>
+    static constexpr int kPiece = 8 * 18;               // bytes of a row's 256 columns
+    static constexpr bool kHasMin = false;              // no per-block offset term
+    static constexpr int kTableBytes = 0;               // no per-warp table of decoded scales
+    static __device__ __forceinline__ void prepare(uint32_t, uint32_t, int) {}
+    template <int U, int BLK, int ROW>
     static __device__ __forceinline__ void block(uint32_t wt, uint32_t (&p)[4]) {
+        constexpr int OFF = ROW + 36 * U;               // the two-block unit
         uint32_t q;
         if (BLK == 0)                                   // quants at bytes 2..17: word t straddles two words
             q = __byte_perm(lds32<OFF>(wt), lds32<OFF + 4>(wt), 0x5432u);
@@ -186,20 +197,27 @@ struct MmaQ40 {
         p[2] = sub_bf16x2(bytes_to_bf16_128_plus<0>(hi), bias);
         p[3] = sub_bf16x2(bytes_to_bf16_128_plus<2>(hi), bias);
     }
-    // `row` = address of the row's piece (without the lane's 4 t)
-    template <int OFF, int BLK>
-    static __device__ __forceinline__ float scale(uint32_t row) { return lds_half<OFF + 18 * BLK>(row); }
+    // `row` = address of the row's piece (without the lane's 4 t); the block's scale (and offset: none)
+    template <int U, int BLK, int ROW>
+    static __device__ __forceinline__ void scales(uint32_t row, uint32_t, float& d, float& m) {
+        d = lds_half<ROW + 36 * U + 18 * BLK>(row);
+        m = 0.f;
+    }
 };
 
 struct MmaQ80 {
-    static constexpr int kBlockBytes = 34;
+    static constexpr int kPiece = 8 * 34;
+    static constexpr bool kHasMin = false;
+    static constexpr int kTableBytes = 0;
+    static __device__ __forceinline__ void prepare(uint32_t, uint32_t, int) {}
     // An int8 code c as bf16: 0x4300 | (c & 0x7F) is 128 + (c & 0x7F), and 0x4300 | (c & 0x80) is 128 or 256;
     // their difference is c.
     static __device__ __forceinline__ uint32_t pair(uint32_t v) {
         return sub_bf16x2(v & 0xFF7FFF7Fu, v & 0xFF80FF80u);
     }
-    template <int OFF, int BLK>
+    template <int U, int BLK, int ROW>
     static __device__ __forceinline__ void block(uint32_t wt, uint32_t (&p)[4]) {
+        constexpr int OFF = ROW + 68 * U;
         uint32_t qa, qb;                                // quant words t and 4 + t of the block
         if (BLK == 0) {                                 // quants at bytes 2..33
             qa = __byte_perm(lds32<OFF>(wt), lds32<OFF + 4>(wt), 0x5432u);
@@ -213,22 +231,85 @@ struct MmaQ80 {
         p[2] = pair(__byte_perm(qb, 0x43434343u, 0x4140u));
         p[3] = pair(__byte_perm(qb, 0x43434343u, 0x4342u));
     }
-    template <int OFF, int BLK>
-    static __device__ __forceinline__ float scale(uint32_t row) { return lds_half<OFF + 34 * BLK>(row); }
+    template <int U, int BLK, int ROW>
+    static __device__ __forceinline__ void scales(uint32_t row, uint32_t, float& d, float& m) {
+        d = lds_half<ROW + 68 * U + 34 * BLK>(row);
+        m = 0.f;
+    }
+};
+
+// q4_K: a row's 256 columns are one 144-byte super-block {d, dmin (fp16), 12 bytes of 6-bit scales and offsets, 128
+// bytes of nibbles}; sub-blocks 2 U and 2 U + 1 are the low and high nibbles of bytes 32 U .. 32 U + 31, and a weight
+// is d * sc * q - dmin * m.  The kernel multiplies the codes q (exact in bf16) and applies d * sc to the sum and
+// dmin * m to the sum of the sub-block's activations, like the fp32-activation streaming family: an activation that
+// is huge beside its neighbours and meets a weight near zero leaves an absolute error (the extra term E of the
+// accuracy statement).  The 6-bit fields are unpacked once per warp and stage into a table of (d * sc, dmin * m).
+struct MmaQ4K {
+    static constexpr int kPiece = 144;
+    static constexpr bool kHasMin = true;
+    static constexpr int kTableBytes = 16 * 8 * 8;      // per warp: 16 rows x 8 sub-blocks x (d * sc, dmin * m)
+    // `rows` = address of the warp's first row piece of the stage, `tab` = the warp's table; lane: row lane / 2,
+    // sub-blocks 4 (lane % 2) .. + 3
+    static __device__ __forceinline__ void prepare(uint32_t rows, uint32_t tab, int lane) {
+        const uint32_t row = rows + (uint32_t)(lane >> 1) * kPiece;
+        const uint32_t dd = lds32<0>(row), w0 = lds32<4>(row), w1 = lds32<8>(row), w2 = lds32<12>(row);
+        const float d = __half2float(__ushort_as_half((unsigned short)(dd & 0xFFFFu)));
+        const float dmin = __half2float(__ushort_as_half((unsigned short)(dd >> 16)));
+        const bool upper = lane & 1;
+        const uint32_t out = tab + (uint32_t)(lane >> 1) * 64u + (upper ? 32u : 0u);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            uint32_t sc, mn;
+            if (!upper) {
+                sc = (w0 >> (8 * j)) & 63u;
+                mn = (w1 >> (8 * j)) & 63u;
+            } else {
+                sc = ((w2 >> (8 * j)) & 0xFu) | (((w0 >> (8 * j + 6)) & 3u) << 4);
+                mn = ((w2 >> (8 * j + 4)) & 0xFu) | (((w1 >> (8 * j + 6)) & 3u) << 4);
+            }
+            const float dsc = d * (float)sc, dmn = dmin * (float)mn;
+            asm volatile("st.shared.v2.f32 [%0], {%1, %2};" ::"r"(out + 8u * j), "f"(dsc), "f"(dmn) : "memory");
+        }
+    }
+    template <int U, int BLK, int ROW>
+    static __device__ __forceinline__ void block(uint32_t wt, uint32_t (&p)[4]) {
+        constexpr int OFF = ROW + 16 + 32 * U;          // the 32 bytes of sub-blocks 2 U (low nibbles), 2 U + 1 (high)
+        uint32_t qa = lds32<OFF>(wt), qb = lds32<OFF + 16>(wt);         // bytes 4t .. 4t+3 and 16+4t .. 16+4t+3
+        if (BLK == 1) {
+            qa >>= 4;
+            qb >>= 4;
+        }
+        qa &= 0x0F0F0F0Fu;
+        qb &= 0x0F0F0F0Fu;
+        const uint32_t bias = 0x43004300u;              // (128, 128): (128 + q) - 128 = q, exactly
+        p[0] = sub_bf16x2(bytes_to_bf16_128_plus<0>(qa), bias);
+        p[1] = sub_bf16x2(bytes_to_bf16_128_plus<2>(qa), bias);
+        p[2] = sub_bf16x2(bytes_to_bf16_128_plus<0>(qb), bias);
+        p[3] = sub_bf16x2(bytes_to_bf16_128_plus<2>(qb), bias);
+    }
+    // ROW / kPiece = row of the warp's 16 (g or g + 8 is added by the caller through `tabg`): tab entry of row g
+    template <int U, int BLK, int ROW>
+    static __device__ __forceinline__ void scales(uint32_t, uint32_t tabg, float& d, float& m) {
+        lds_f32x2<(ROW / kPiece) * 64 + 8 * (2 * U + BLK)>(tabg, d, m);
+    }
 };
 
 // One block (32 weights) of the warp's 16 rows against all columns: decode the lane's fragments of rows g and
 // g + 8, six products per group of eight columns into one accumulator, then the block scales in fp32.
 // U = unit of the stage (0..3), BLK = block of the unit; xp[nt][s] = address of the lane's B fragments of plane s,
 // column group nt, at the stage's first column.
+// tabg = the warp's scale table at row g (formats with one); sx = address of the lane's two block sums of the
+// activations, group nt 32 bytes further (formats with an offset term).
 template <class T, int NT, int U, int BLK>
-__device__ __forceinline__ void block_step(uint32_t wt, uint32_t row, const uint32_t (&xp)[NT][3], float (&y)[NT][4]) {
-    constexpr int kPiece = kStageCols / 32 * T::kBlockBytes;
-    constexpr int kUnit = U * 2 * T::kBlockBytes;
+__device__ __forceinline__ void block_step(uint32_t wt, uint32_t row, uint32_t tabg, uint32_t sx,
+                                           const uint32_t (&xp)[NT][3], float (&y)[NT][4]) {
+    constexpr int kPiece = T::kPiece;
     uint32_t a[4], b[4];
-    T::template block<kUnit, BLK>(wt, a);
-    T::template block<kUnit + 8 * kPiece, BLK>(wt, b);
-    const float d0 = T::template scale<kUnit, BLK>(row), d1 = T::template scale<kUnit + 8 * kPiece, BLK>(row);
+    T::template block<U, BLK, 0>(wt, a);
+    T::template block<U, BLK, 8 * kPiece>(wt, b);
+    float d0, d1, m0, m1;
+    T::template scales<U, BLK, 0>(row, tabg, d0, m0);
+    T::template scales<U, BLK, 8 * kPiece>(row, tabg, d1, m1);
     constexpr int kX = 2 * (64 * U + 32 * BLK);          // bytes into a plane's column
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) {
@@ -247,6 +328,18 @@ __device__ __forceinline__ void block_step(uint32_t wt, uint32_t row, const uint
         y[nt][1] = fmaf(d0, c[1], y[nt][1]);
         y[nt][2] = fmaf(d1, c[2], y[nt][2]);
         y[nt][3] = fmaf(d1, c[3], y[nt][3]);
+        if constexpr (T::kHasMin) {
+            // minus the block's offset times the sum of its activations (columns 2 t and 2 t + 1 of the group)
+            float s0, s1;
+            if (nt == 0)
+                lds_f32x2<kSxBlockBytes * (2 * U + BLK)>(sx, s0, s1);
+            else
+                lds_f32x2<kSxBlockBytes * (2 * U + BLK) + 32>(sx, s0, s1);
+            y[nt][0] = fmaf(-m0, s0, y[nt][0]);
+            y[nt][1] = fmaf(-m0, s1, y[nt][1]);
+            y[nt][2] = fmaf(-m1, s0, y[nt][2]);
+            y[nt][3] = fmaf(-m1, s1, y[nt][3]);
+        }
     }
 }
 
@@ -314,7 +407,7 @@ __global__ void __launch_bounds__(kMmaThreads, kCtasPerSm) matvec_mma_kernel(con
     uint64_t* empty = full + kMaxRing;                                // [kMaxRing]
     volatile int* stop = reinterpret_cast<volatile int*>(smem + 64);  // set when a wait gave up
     constexpr int NB = 8 * NT;                                        // columns held (beyond the batch: zeros)
-    constexpr int kPiece = kStageCols / 32 * T::kBlockBytes;          // bytes of a row's share of a stage
+    constexpr int kPiece = T::kPiece;                                 // bytes of a row's share of a stage
     constexpr int kStageBytes = kStageRows * kPiece;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -497,6 +590,16 @@ __global__ void __launch_bounds__(kMmaThreads, kCtasPerSm) matvec_mma_kernel(con
                         split3(v[q][nt].y, h[0][1], h[1][1], h[2][1]);
                         split3(v[q][nt].z, h[0][2], h[1][2], h[2][2]);
                         split3(v[q][nt].w, h[0][3], h[1][3], h[2][3]);
+                        if constexpr (T::kHasMin) {
+                            // sum of each block of 32 activations (eight consecutive lanes hold one), for the
+                            // formats with a per-block offset: [block of the chunk][column]
+                            float sum = (v[q][nt].x + v[q][nt].y) + (v[q][nt].z + v[q][nt].w);
+                            sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+                            sum += __shfl_xor_sync(0xffffffffu, sum, 2);
+                            sum += __shfl_xor_sync(0xffffffffu, sum, 4);
+                            if ((lane & 7) == 0)
+                                *reinterpret_cast<float*>(smem + p.sx_off + (size_t)(k4 >> 3) * kSxBlockBytes + 4 * b) = sum;
+                        }
                         const int slot4 = (k4 & ~7) + 2 * (k4 & 3) + ((k4 >> 2) & 1);    // quad of slots the quad of k goes to
                         const uint32_t dst = xs + b * x_pitch + 8u * slot4;
 #pragma unroll
@@ -518,20 +621,26 @@ __global__ void __launch_bounds__(kMmaThreads, kCtasPerSm) matvec_mma_kernel(con
         const int64_t r0 = (int64_t)(rs - mat.rs_begin) * kStageRows;
         if (r0 + 16 * warp < mat.rows) {
             const uint32_t row = wrow + (uint32_t)slot * kStageBytes, wt = row + 4u * t;
+            const uint32_t tab = smem_u32(smem + p.tab_off) + (uint32_t)warp * T::kTableBytes, tabg = tab + 64u * g;
+            const uint32_t sx = smem_u32(smem + p.sx_off) + (uint32_t)(8 * j) * kSxBlockBytes + 8u * t;
+            if constexpr (T::kTableBytes > 0) {
+                T::prepare(row - (uint32_t)g * kPiece, tab, lane);
+                __syncwarp();
+            }
             uint32_t xp[NT][3];
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
                 for (int s = 0; s < 3; ++s)
                     xp[nt][s] = xlane + 2u * (uint32_t)(j * kStageCols) + s * plane_pitch + nt * 8 * x_pitch;
-            block_step<T, NT, 0, 0>(wt, row, xp, y);
-            block_step<T, NT, 0, 1>(wt, row, xp, y);
-            block_step<T, NT, 1, 0>(wt, row, xp, y);
-            block_step<T, NT, 1, 1>(wt, row, xp, y);
-            block_step<T, NT, 2, 0>(wt, row, xp, y);
-            block_step<T, NT, 2, 1>(wt, row, xp, y);
-            block_step<T, NT, 3, 0>(wt, row, xp, y);
-            block_step<T, NT, 3, 1>(wt, row, xp, y);
+            block_step<T, NT, 0, 0>(wt, row, tabg, sx, xp, y);
+            block_step<T, NT, 0, 1>(wt, row, tabg, sx, xp, y);
+            block_step<T, NT, 1, 0>(wt, row, tabg, sx, xp, y);
+            block_step<T, NT, 1, 1>(wt, row, tabg, sx, xp, y);
+            block_step<T, NT, 2, 0>(wt, row, tabg, sx, xp, y);
+            block_step<T, NT, 2, 1>(wt, row, tabg, sx, xp, y);
+            block_step<T, NT, 3, 0>(wt, row, tabg, sx, xp, y);
+            block_step<T, NT, 3, 1>(wt, row, tabg, sx, xp, y);
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(&empty[slot]);
@@ -608,26 +717,31 @@ int mma_sm_count() {
 
 // Shared-memory plan of a launch: the largest chunk (1024, 512, 256 columns) that divides cols and leaves room
 // for at least two stages.  Returns false if nothing fits.
-bool mma_plan(int fmt, int64_t cols, int nt, int& chunk_cols, int& ring, size_t& x_bytes, size_t& stage_bytes) {
-    const int block_bytes = fmt == LW_Q4_0 ? 18 : 34;
-    stage_bytes = (size_t)kStageRows * (kStageCols / 32) * block_bytes;
-    const size_t budget = kSmemPerCta - kMmaHeader;
-    for (int kx = 1024; kx >= 256; kx /= 2) {
-        if (cols % kx != 0) continue;
-        x_bytes = (size_t)3 * 8 * nt * (2 * kx + kXPad);
-        if (x_bytes + 2 * stage_bytes > budget) continue;
-        size_t n = (budget - x_bytes) / stage_bytes;
-        ring = (int)(n > (size_t)kMaxRing ? kMaxRing : n);
-        chunk_cols = kx;
-        return true;
-    }
+bool mma_plan(int fmt, int64_t cols, int nt, int& chunk_cols, int& ring, size_t& x_bytes, size_t& stage_bytes,
+              size_t& extra_bytes) {
+    const int piece = fmt == LW_Q8_0 ? MmaQ80::kPiece : (fmt == LW_Q4_0 ? MmaQ40::kPiece : MmaQ4K::kPiece);
+    stage_bytes = (size_t)kStageRows * piece;
+    // q4_K: block sums of the activations (64 bytes per block of a chunk of up to 1024 columns) and the warps' tables
+    extra_bytes = fmt == LW_Q4_K ? (size_t)(1024 / 32) * kSxBlockBytes + (size_t)kMmaWarps * MmaQ4K::kTableBytes : 0;
+    const size_t budget = kSmemPerCta - kMmaHeader - extra_bytes;
+    // the largest chunk that leaves room for three stages, else for two
+    for (size_t min_ring = 3; min_ring >= 2; --min_ring)
+        for (int kx = 1024; kx >= 256; kx /= 2) {
+            if (cols % kx != 0) continue;
+            x_bytes = (size_t)3 * 8 * nt * (2 * kx + kXPad);
+            if (x_bytes + min_ring * stage_bytes > budget) continue;
+            size_t n = (budget - x_bytes) / stage_bytes;
+            ring = (int)(n > (size_t)kMaxRing ? kMaxRing : n);
+            chunk_cols = kx;
+            return true;
+        }
     return false;
 }
 
 }  // namespace
 
 bool matvec_mma_supported(int fmt, int64_t rows, int64_t cols, int batch) {
-    if (fmt != LW_Q4_0 && fmt != LW_Q8_0) return false;
+    if (fmt != LW_Q4_0 && fmt != LW_Q8_0 && fmt != LW_Q4_K) return false;
     if (batch < 2 || batch > 16) return false;
     if (cols % kStageCols != 0) return false;
     return rows >= 1 && rows <= (int64_t)1 << 30;
@@ -654,6 +768,17 @@ int launch_matvec_mma_group(int fmt, int64_t cols, int n_items, const void* cons
                             cudaStream_t stream) {
     int* fault = device_fault_word();
     if (!fault) return (int)cudaErrorInvalidValue;
+    {
+        // The grid barrier of the self-clearing form is one pair of words per device: it relies on two such
+        // launches never running at the same time, which holds because each needs every SM to itself (cooperative
+        // launch, one CTA per SM, more than half an SM's shared memory per CTA).  Should a plan ever need less, take
+        // the clearing kernel instead.
+        int cc = 0, rg = 0;
+        size_t xb = 0, sb = 0, eb = 0;
+        if (!mma_plan(fmt, cols, batch > 8 ? 2 : 1, cc, rg, xb, sb, eb)) return (int)cudaErrorInvalidValue;
+        if (2 * ((kMmaHeader + xb + eb + 127) / 128 * 128 + (size_t)rg * sb + 1024) <= 228 * 1024 || kCtasPerSm != 1)
+            self_clear = false;
+    }
     unsigned* grid_bar = nullptr;
     if (self_clear && cudaGetSymbolAddress(reinterpret_cast<void**>(&grid_bar), g_mma_grid_barrier) != cudaSuccess)
         return (int)cudaErrorInvalidValue;
@@ -678,8 +803,8 @@ int launch_matvec_mma_group(int fmt, int64_t cols, int n_items, const void* cons
     }
     const int nt = batch > 8 ? 2 : 1;
     MmaParams p{};
-    size_t x_bytes = 0, stage_bytes = 0;
-    if (!mma_plan(fmt, cols, nt, p.chunk_cols, p.ring, x_bytes, stage_bytes)) return (int)cudaErrorInvalidValue;
+    size_t x_bytes = 0, stage_bytes = 0, extra_bytes = 0;
+    if (!mma_plan(fmt, cols, nt, p.chunk_cols, p.ring, x_bytes, stage_bytes, extra_bytes)) return (int)cudaErrorInvalidValue;
     alignas(64) MmaMaps maps;
     const int64_t row_bytes = (int64_t)lw_row_bytes(fmt, cols);
     int rs = 0;
@@ -704,7 +829,9 @@ int launch_matvec_mma_group(int fmt, int64_t cols, int n_items, const void* cons
     p.self_clear = self_clear ? 1 : 0;
     p.grid_bar = grid_bar;
     p.x_off = kMmaHeader;
-    p.w_off = (uint32_t)((kMmaHeader + x_bytes + 127) / 128 * 128);
+    p.sx_off = (uint32_t)(kMmaHeader + x_bytes);
+    p.tab_off = p.sx_off + (uint32_t)(fmt == LW_Q4_K ? (1024 / 32) * kSxBlockBytes : 0);
+    p.w_off = (uint32_t)((kMmaHeader + x_bytes + extra_bytes + 127) / 128 * 128);
     const size_t smem_bytes = p.w_off + (size_t)p.ring * stage_bytes;
     const int64_t n_stages = (cols / kStageCols) * (int64_t)rs;
     int grid = kCtasPerSm * mma_sm_count();
@@ -712,6 +839,9 @@ int launch_matvec_mma_group(int fmt, int64_t cols, int n_items, const void* cons
     if (fmt == LW_Q4_0)
         return nt == 1 ? launch_mma<MmaQ40, 1>(p, maps, grid, smem_bytes, overlap != 0, stream)
                        : launch_mma<MmaQ40, 2>(p, maps, grid, smem_bytes, overlap != 0, stream);
+    if (fmt == LW_Q4_K)
+        return nt == 1 ? launch_mma<MmaQ4K, 1>(p, maps, grid, smem_bytes, overlap != 0, stream)
+                       : launch_mma<MmaQ4K, 2>(p, maps, grid, smem_bytes, overlap != 0, stream);
     return nt == 1 ? launch_mma<MmaQ80, 1>(p, maps, grid, smem_bytes, overlap != 0, stream)
                    : launch_mma<MmaQ80, 2>(p, maps, grid, smem_bytes, overlap != 0, stream);
 }

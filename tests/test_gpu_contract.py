@@ -131,6 +131,31 @@ def test_batched_kernels_need_no_extra_term(fmt, kernel):
     assert (np.abs(y.astype(np.float64) - y_ref)[finite] <= (RTOL * s_ref + ATOL)[finite]).all()
 
 
+def test_q4_K_on_the_tensor_cores_stays_inside_the_stated_bound():
+    # q4_K in the batched tensor-core kernel applies the sub-block offsets to sums of activations, like the
+    # fp32-activation streaming family: the header gives it the extra term with c = 2^-18, asserted here on the
+    # adversarial activations (eight columns, each with its own outliers), and a non-finite activation stays in its
+    # column
+    fmt, rows, cols, batch = lw.Q4_K, 48, 4096, 8
+    cols_x = []
+    for b in range(batch):
+        blocks, X = _adversarial(fmt, rows, cols, seed=90 + fmt, zero_rest_of_vector=bool(b & 1))
+        cols_x.append(X[0] * (1.0 + b))
+    X = np.stack(cols_x).astype(np.float32)
+    y_ref, s_ref = oracle.matvec(fmt, blocks, rows, cols, X, batch)
+    lw.set_variant(lw.VARIANT_MMA)
+    assert lw.query_variant(fmt, rows, cols, batch) == lw.VARIANT_MMA
+    y = _run(fmt, blocks, rows, cols, X, lw.VARIANT_MMA, batch)
+    for b in range(batch):
+        bound = RTOL * s_ref[b] + ATOL + _extra_term(fmt, blocks, rows, cols, X[b:b + 1], 2.0 ** -18)[0]
+        worst = float((np.abs(y[b].astype(np.float64) - y_ref[b]) / bound).max())
+        assert worst <= 1.0, "column %d: error / bound = %.3g" % (b, worst)
+    Xb = X.copy()
+    Xb[3, 100] = np.nan
+    y = _run(fmt, blocks, rows, cols, Xb, lw.VARIANT_MMA, batch)
+    assert not np.isfinite(y[3]).any() and np.isfinite(np.delete(y, 3, axis=0)).all()
+
+
 @pytest.mark.parametrize("variant", ALL_VARIANTS)
 @pytest.mark.parametrize("fmt", FMTS)
 def test_non_finite_activations_reach_the_output(fmt, variant):

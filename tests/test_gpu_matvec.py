@@ -79,13 +79,13 @@ def test_matvec_tile_kernel(fmt, batch, rows, cols):
     check_matvec(y, y_ref, s_ref, "tile fmt %d %dx%d batch %d" % (fmt, rows, cols, batch))
 
 
-@pytest.mark.parametrize("fmt", [lw.Q8_0, lw.Q4_0])
+@pytest.mark.parametrize("fmt", [lw.Q8_0, lw.Q4_0, lw.Q4_K])
 @pytest.mark.parametrize("batch", [2, 3, 7, 8, 9, 16])
 @pytest.mark.parametrize("rows,cols", [(1, 256), (15, 512), (16, 1024), (17, 768), (255, 2048), (256, 1024), (257, 4096),
                                        (333, 3072), (1000, 14336), (4096, 1280), (70000, 1024)])
 def test_matvec_mma_kernel(fmt, batch, rows, cols):
-    # the batched tensor-core kernel (AUTO's choice for q8_0 / q4_0 from three columns on when cols is a multiple of
-    # 256): ragged row counts around its 16-row fragments and 256-row stages, chunks of 256 / 512 / 1024 columns,
+    # the batched tensor-core kernel (AUTO's choice for q8_0 / q4_0 / q4_K from three columns on when cols is a
+    # multiple of 256): ragged row counts around its 16-row fragments and 256-row stages, chunks of 256 / 512 / 1024 columns,
     # one and two groups of eight columns, more stages than CTAs (70000 rows) and fewer (1 row)
     lw.set_variant(lw.VARIANT_AUTO)
     assert lw.query_variant(fmt, rows, cols, batch) == (lw.VARIANT_MMA if batch >= 3 else lw.VARIANT_IDOT)
@@ -99,7 +99,7 @@ def test_matvec_mma_kernel(fmt, batch, rows, cols):
 
 
 @pytest.mark.parametrize("overlap", [0, 1, 2])
-@pytest.mark.parametrize("fmt", [lw.Q8_0, lw.Q4_0])
+@pytest.mark.parametrize("fmt", [lw.Q8_0, lw.Q4_0, lw.Q4_K])
 def test_matvec_mma_launch_modes(fmt, overlap):
     # the two ways the tensor-core kernel gets a cleared Y: one cooperative launch whose CTAs clear it and meet at a
     # grid barrier (no overlap), or a clearing kernel chained to it by programmatic dependent launch (overlap 1;

@@ -131,7 +131,7 @@ def test_variant_controls():
     assert lw.query_variant(lw.Q4_K, 4096, 4096, 1) == lw.VARIANT_IDOT
     assert lw.query_variant(lw.F16, 4096, 4096, 1) == lw.VARIANT_STREAM
     assert lw.query_variant(lw.Q4_K, 4096, 4096, 2) == lw.VARIANT_IDOT       # one integer-dot pass per column
-    assert lw.query_variant(lw.Q4_0, 4096, 4096, 16) == lw.VARIANT_MMA       # tensor-core kernel: q8_0 / q4_0, cols % 256 == 0
+    assert lw.query_variant(lw.Q4_0, 4096, 4096, 16) == lw.VARIANT_MMA       # tensor-core kernel: q8_0 / q4_0 / q4_K, cols % 256 == 0
     assert lw.query_variant(lw.Q8_0, 128256, 4096, 3) == lw.VARIANT_MMA
     assert lw.query_variant(lw.Q8_0, 128256, 4096, 2) == lw.VARIANT_IDOT        # two columns: one pass per column
     assert lw.query_variant(lw.Q4_0, 4096, 4096 + 512, 16) == lw.VARIANT_MMA
@@ -141,7 +141,8 @@ def test_variant_controls():
     assert lw.query_variant(lw.Q4_0, 4096, 4096 + 512, 16) != lw.VARIANT_TILE
     lw.set_variant(lw.VARIANT_MMA)
     assert lw.query_variant(lw.Q4_0, 4096, 4096, 2) == lw.VARIANT_MMA
-    assert lw.query_variant(lw.Q4_K, 4096, 4096, 8) != lw.VARIANT_MMA
+    assert lw.query_variant(lw.Q4_K, 4096, 4096, 8) == lw.VARIANT_MMA         # q4_K as well (with the extra term E)
+    assert lw.query_variant(lw.Q6_K, 4096, 4096, 8) != lw.VARIANT_MMA
     assert lw.query_variant(lw.Q4_0, 4096, 4096, 1) == lw.VARIANT_IDOT        # batch 1: falls back
     lw.set_variant(lw.VARIANT_AUTO)
     assert lw.query_variant(lw.Q4_1, 4096, 4096, 16) == lw.VARIANT_IDOT
