@@ -724,17 +724,17 @@ bool mma_plan(int fmt, int64_t cols, int nt, int& chunk_cols, int& ring, size_t&
     // q4_K: block sums of the activations (64 bytes per block of a chunk of up to 1024 columns) and the warps' tables
     extra_bytes = fmt == LW_Q4_K ? (size_t)(1024 / 32) * kSxBlockBytes + (size_t)kMmaWarps * MmaQ4K::kTableBytes : 0;
     const size_t budget = kSmemPerCta - kMmaHeader - extra_bytes;
-    // the largest chunk that leaves room for three stages, else for two
-    for (size_t min_ring = 3; min_ring >= 2; --min_ring)
-        for (int kx = 1024; kx >= 256; kx /= 2) {
-            if (cols % kx != 0) continue;
-            x_bytes = (size_t)3 * 8 * nt * (2 * kx + kXPad);
-            if (x_bytes + min_ring * stage_bytes > budget) continue;
-            size_t n = (budget - x_bytes) / stage_bytes;
-            ring = (int)(n > (size_t)kMaxRing ? kMaxRing : n);
-            chunk_cols = kx;
-            return true;
-        }
+    // the largest chunk that leaves room for two stages (q8_0, 458752 x 4096, 8 columns: 0.40 ms with chunks of
+    // 1024 columns and two 68 KB stages against 0.49 ms with chunks of 256 and three)
+    for (int kx = 1024; kx >= 256; kx /= 2) {
+        if (cols % kx != 0) continue;
+        x_bytes = (size_t)3 * 8 * nt * (2 * kx + kXPad);
+        if (x_bytes + 2 * stage_bytes > budget) continue;
+        size_t n = (budget - x_bytes) / stage_bytes;
+        ring = (int)(n > (size_t)kMaxRing ? kMaxRing : n);
+        chunk_cols = kx;
+        return true;
+    }
     return false;
 }
 
