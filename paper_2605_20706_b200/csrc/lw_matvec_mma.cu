@@ -1,4 +1,4 @@
-// Batched mat-vec on the tensor cores (batch 2..16; q4_0, q8_0 and q4_K) [paper Sec 3.2: from a handful of columns on
+// Batched mat-vec on the tensor cores (batch 2..16; q4_0, q8_0, q4_K and q5_K) [paper Sec 3.2: from a handful of columns on
 // the mat-vec turns into a small mat-mat product, a dense contraction; Sec 3.3: one decode routine per format
 // spliced into a common skeleton].
 //
@@ -288,6 +288,57 @@ struct MmaQ4K {
         p[3] = sub_bf16x2(bytes_to_bf16_128_plus<2>(qb), bias);
     }
     // ROW / kPiece = row of the warp's 16 (g or g + 8 is added by the caller through `tabg`): tab entry of row g
+    template <int U, int BLK, int ROW>
+    static __device__ __forceinline__ void scales(uint32_t, uint32_t tabg, float& d, float& m) {
+        lds_f32x2<(ROW / kPiece) * 64 + 8 * (2 * U + BLK)>(tabg, d, m);
+    }
+};
+
+// q5_K: q4_K's layout with 32 bytes of fifth bits between the scales and the nibbles (176 bytes per 256 weights): bit
+// s of byte l is the high bit of weight l of sub-block s, so a code is 0..31 -- still exact in bf16.
+struct MmaQ5K {
+    static constexpr int kPiece = 176;
+    static constexpr bool kHasMin = true;
+    static constexpr int kTableBytes = MmaQ4K::kTableBytes;
+    static __device__ __forceinline__ void prepare(uint32_t rows, uint32_t tab, int lane) {
+        // the same header {d, dmin, 12 bytes of 6-bit fields} at the same offsets, rows 176 bytes apart
+        const uint32_t row = rows + (uint32_t)(lane >> 1) * kPiece;
+        const uint32_t dd = lds32<0>(row), w0 = lds32<4>(row), w1 = lds32<8>(row), w2 = lds32<12>(row);
+        const float d = __half2float(__ushort_as_half((unsigned short)(dd & 0xFFFFu)));
+        const float dmin = __half2float(__ushort_as_half((unsigned short)(dd >> 16)));
+        const bool upper = lane & 1;
+        const uint32_t out = tab + (uint32_t)(lane >> 1) * 64u + (upper ? 32u : 0u);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            uint32_t sc, mn;
+            if (!upper) {
+                sc = (w0 >> (8 * j)) & 63u;
+                mn = (w1 >> (8 * j)) & 63u;
+            } else {
+                sc = ((w2 >> (8 * j)) & 0xFu) | (((w0 >> (8 * j + 6)) & 3u) << 4);
+                mn = ((w2 >> (8 * j + 4)) & 0xFu) | (((w1 >> (8 * j + 6)) & 3u) << 4);
+            }
+            const float dsc = d * (float)sc, dmn = dmin * (float)mn;
+            asm volatile("st.shared.v2.f32 [%0], {%1, %2};" ::"r"(out + 8u * j), "f"(dsc), "f"(dmn) : "memory");
+        }
+    }
+    template <int U, int BLK, int ROW>
+    static __device__ __forceinline__ void block(uint32_t wt, uint32_t (&p)[4]) {
+        constexpr int S = 2 * U + BLK;                  // sub-block = bit of the fifth-bit bytes
+        uint32_t qa = lds32<ROW + 48 + 32 * U>(wt), qb = lds32<ROW + 48 + 32 * U + 16>(wt);
+        const uint32_t ha = lds32<ROW + 16>(wt), hb = lds32<ROW + 32>(wt);   // fifth bits of weights 4t.. and 16+4t..
+        if (BLK == 1) {
+            qa >>= 4;
+            qb >>= 4;
+        }
+        qa = (qa & 0x0F0F0F0Fu) | (((ha >> S) & 0x01010101u) << 4);
+        qb = (qb & 0x0F0F0F0Fu) | (((hb >> S) & 0x01010101u) << 4);
+        const uint32_t bias = 0x43004300u;              // (128, 128): (128 + q) - 128 = q, exactly
+        p[0] = sub_bf16x2(bytes_to_bf16_128_plus<0>(qa), bias);
+        p[1] = sub_bf16x2(bytes_to_bf16_128_plus<2>(qa), bias);
+        p[2] = sub_bf16x2(bytes_to_bf16_128_plus<0>(qb), bias);
+        p[3] = sub_bf16x2(bytes_to_bf16_128_plus<2>(qb), bias);
+    }
     template <int U, int BLK, int ROW>
     static __device__ __forceinline__ void scales(uint32_t, uint32_t tabg, float& d, float& m) {
         lds_f32x2<(ROW / kPiece) * 64 + 8 * (2 * U + BLK)>(tabg, d, m);
@@ -719,10 +770,12 @@ int mma_sm_count() {
 // for at least two stages.  Returns false if nothing fits.
 bool mma_plan(int fmt, int64_t cols, int nt, int& chunk_cols, int& ring, size_t& x_bytes, size_t& stage_bytes,
               size_t& extra_bytes) {
-    const int piece = fmt == LW_Q8_0 ? MmaQ80::kPiece : (fmt == LW_Q4_0 ? MmaQ40::kPiece : MmaQ4K::kPiece);
+    const int piece = fmt == LW_Q8_0 ? MmaQ80::kPiece
+                                     : fmt == LW_Q4_0 ? MmaQ40::kPiece : fmt == LW_Q4_K ? MmaQ4K::kPiece : MmaQ5K::kPiece;
     stage_bytes = (size_t)kStageRows * piece;
     // q4_K: block sums of the activations (64 bytes per block of a chunk of up to 1024 columns) and the warps' tables
-    extra_bytes = fmt == LW_Q4_K ? (size_t)(1024 / 32) * kSxBlockBytes + (size_t)kMmaWarps * MmaQ4K::kTableBytes : 0;
+    extra_bytes = (fmt == LW_Q4_K || fmt == LW_Q5_K)
+                      ? (size_t)(1024 / 32) * kSxBlockBytes + (size_t)kMmaWarps * MmaQ4K::kTableBytes : 0;
     const size_t budget = kSmemPerCta - kMmaHeader - extra_bytes;
     // the largest chunk that leaves room for two stages (q8_0, 458752 x 4096, 8 columns: 0.40 ms with chunks of
     // 1024 columns and two 68 KB stages against 0.49 ms with chunks of 256 and three)
@@ -741,7 +794,7 @@ bool mma_plan(int fmt, int64_t cols, int nt, int& chunk_cols, int& ring, size_t&
 }  // namespace
 
 bool matvec_mma_supported(int fmt, int64_t rows, int64_t cols, int batch) {
-    if (fmt != LW_Q4_0 && fmt != LW_Q8_0 && fmt != LW_Q4_K) return false;
+    if (fmt != LW_Q4_0 && fmt != LW_Q8_0 && fmt != LW_Q4_K && fmt != LW_Q5_K) return false;
     if (batch < 2 || batch > 16) return false;
     if (cols % kStageCols != 0) return false;
     return rows >= 1 && rows <= (int64_t)1 << 30;
@@ -830,7 +883,7 @@ int launch_matvec_mma_group(int fmt, int64_t cols, int n_items, const void* cons
     p.grid_bar = grid_bar;
     p.x_off = kMmaHeader;
     p.sx_off = (uint32_t)(kMmaHeader + x_bytes);
-    p.tab_off = p.sx_off + (uint32_t)(fmt == LW_Q4_K ? (1024 / 32) * kSxBlockBytes : 0);
+    p.tab_off = p.sx_off + (uint32_t)((fmt == LW_Q4_K || fmt == LW_Q5_K) ? (1024 / 32) * kSxBlockBytes : 0);
     p.w_off = (uint32_t)((kMmaHeader + x_bytes + extra_bytes + 127) / 128 * 128);
     const size_t smem_bytes = p.w_off + (size_t)p.ring * stage_bytes;
     const int64_t n_stages = (cols / kStageCols) * (int64_t)rs;
@@ -842,6 +895,9 @@ int launch_matvec_mma_group(int fmt, int64_t cols, int n_items, const void* cons
     if (fmt == LW_Q4_K)
         return nt == 1 ? launch_mma<MmaQ4K, 1>(p, maps, grid, smem_bytes, overlap != 0, stream)
                        : launch_mma<MmaQ4K, 2>(p, maps, grid, smem_bytes, overlap != 0, stream);
+    if (fmt == LW_Q5_K)
+        return nt == 1 ? launch_mma<MmaQ5K, 1>(p, maps, grid, smem_bytes, overlap != 0, stream)
+                       : launch_mma<MmaQ5K, 2>(p, maps, grid, smem_bytes, overlap != 0, stream);
     return nt == 1 ? launch_mma<MmaQ80, 1>(p, maps, grid, smem_bytes, overlap != 0, stream)
                    : launch_mma<MmaQ80, 2>(p, maps, grid, smem_bytes, overlap != 0, stream);
 }

@@ -131,12 +131,13 @@ def test_batched_kernels_need_no_extra_term(fmt, kernel):
     assert (np.abs(y.astype(np.float64) - y_ref)[finite] <= (RTOL * s_ref + ATOL)[finite]).all()
 
 
-def test_q4_K_on_the_tensor_cores_stays_inside_the_stated_bound():
-    # q4_K in the batched tensor-core kernel applies the sub-block offsets to sums of activations, like the
-    # fp32-activation streaming family: the header gives it the extra term with c = 2^-18, asserted here on the
+@pytest.mark.parametrize("fmt", [lw.Q4_K, lw.Q5_K])
+def test_k_quants_on_the_tensor_cores_stay_inside_the_stated_bound(fmt):
+    # q4_K / q5_K in the batched tensor-core kernel apply the sub-block offsets to sums of activations, like the
+    # fp32-activation streaming family: the header gives them the extra term with c = 2^-18, asserted here on the
     # adversarial activations (eight columns, each with its own outliers), and a non-finite activation stays in its
     # column
-    fmt, rows, cols, batch = lw.Q4_K, 48, 4096, 8
+    rows, cols, batch = 48, 4096, 8
     cols_x = []
     for b in range(batch):
         blocks, X = _adversarial(fmt, rows, cols, seed=90 + fmt, zero_rest_of_vector=bool(b & 1))
