@@ -361,7 +361,10 @@ int lw_probe_read(const void* src, int64_t bytes, void* stream);
  * next batch-1 lw_matvec of a q4_K matrix that takes the streaming kernel (a separate build of it: the kernels
  * of ordinary calls carry no trace of this aid) never requests the copy of the u-th row unit of each CTA: nothing is in flight for it, the wait for it runs out after its limit (about 0.1 s), the kernel
  * records a fault, requests nothing further and returns; the rows of that unit and of the units after it are
- * left unwritten.  The request is consumed by that one launch; u < 0 cancels it.  Always returns LW_OK. */
+ * left unwritten.  The batched tensor-core kernel has the same aid for q4_0 with up to 8 columns: the launch that
+ * consumes the request asks for no copy from each CTA's u-th stage on, the wait for that stage runs out, the fault
+ * is recorded and the kernel returns (its results are meaningless).  The request is consumed by the first launch of
+ * either kind; u < 0 cancels it.  Always returns LW_OK. */
 int lw_debug_drop_copy(int unit);
 
 #ifdef __cplusplus

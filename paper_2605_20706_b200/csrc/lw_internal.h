@@ -65,6 +65,7 @@ void set_shape_tuning(int fmt, int64_t rows, int64_t cols, int worker_groups, in
 void clear_shape_tuning();
 // Testing aid: the next single-matrix streaming launch never requests the copy of pool unit `unit` (< 0: none).
 void set_drop_unit(int unit);
+int take_drop_unit();     // the pending request (-1: none), consumed
 bool stream_plan_info(int fmt, int64_t rows, int64_t cols, int* groups, int* stages, int* stage_rows, int* stage_bytes,
                       int* grid, int* smem_bytes);
 // Decode attention over a quantised KV cache: shape check, parts the positions are cut into, bytes of

@@ -103,6 +103,7 @@ struct MmaParams {
     unsigned* grid_bar;   // {arrival count, generation} of that barrier, owned by the library
     uint32_t x_off, w_off;
     uint32_t sx_off, tab_off;   // block sums of the activations and the warps' scale tables (formats that need them)
+    int drop_stage;       // testing aid (separate kernel build): the CTA's stage from which on no copy is requested
 };
 
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
@@ -450,7 +451,9 @@ struct Cursor {
     }
 };
 
-template <class T, int NT>
+// DROP: a build for lw_debug_drop_copy (the producer requests nothing from stage p.drop_stage on, so the wait for
+// that stage runs out); the kernels of ordinary calls carry none of it.
+template <class T, int NT, bool DROP = false>
 __global__ void __launch_bounds__(kMmaThreads, kCtasPerSm) matvec_mma_kernel(const __grid_constant__ MmaParams p,
                                                                              const __grid_constant__ MmaMaps maps) {
     extern __shared__ __align__(128) uint8_t smem[];
@@ -499,6 +502,9 @@ __global__ void __launch_bounds__(kMmaThreads, kCtasPerSm) matvec_mma_kernel(con
         int n = 0;
         for (; n < count; ++n, cur.step(p, spc, ring)) {
             if (*stop) break;
+            if constexpr (DROP) {
+                if (n >= p.drop_stage) break;
+            }
             if (n >= ring && !mbar_wait_bounded(&empty[cur.slot], cur.parity ^ 1u)) {   // the slot's previous use
                 atomicExch(p.fault, (int)FAULT_BULK_WAIT_TIMEOUT);
                 *stop = 1;
@@ -699,7 +705,7 @@ __global__ void __launch_bounds__(kMmaThreads, kCtasPerSm) matvec_mma_kernel(con
     if (cur_rs >= 0) flush();
 }
 
-template <class T, int NT>
+template <class T, int NT, bool DROP = false>
 int launch_mma(const MmaParams& p, const MmaMaps& maps, int grid, size_t smem_bytes, bool overlap,
                cudaStream_t stream) {
     // self-clearing launches are cooperative (their CTAs wait for one another) and ordinary in stream order
@@ -708,7 +714,7 @@ int launch_mma(const MmaParams& p, const MmaMaps& maps, int grid, size_t smem_by
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return (int)e;
     if (dev < 0 || dev >= 64 || !attr_set[dev]) {
-        e = cudaFuncSetAttribute(matvec_mma_kernel<T, NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemPerCta);
+        e = cudaFuncSetAttribute(matvec_mma_kernel<T, NT, DROP>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemPerCta);
         if (e != cudaSuccess) return (int)e;
         if (dev >= 0 && dev < 64) attr_set[dev] = true;
     }
@@ -727,7 +733,7 @@ int launch_mma(const MmaParams& p, const MmaMaps& maps, int grid, size_t smem_by
     }
     cfg.attrs = attr;
     cfg.numAttrs = (p.self_clear || overlap) ? 1 : 0;
-    return (int)cudaLaunchKernelEx(&cfg, matvec_mma_kernel<T, NT>, p, maps);
+    return (int)cudaLaunchKernelEx(&cfg, matvec_mma_kernel<T, NT, DROP>, p, maps);
 }
 
 // cuTensorMapEncodeTiled through the runtime's driver entry point lookup (no link against the driver library)
@@ -889,6 +895,15 @@ int launch_matvec_mma_group(int fmt, int64_t cols, int n_items, const void* cons
     const int64_t n_stages = (cols / kStageCols) * (int64_t)rs;
     int grid = kCtasPerSm * mma_sm_count();
     if ((int64_t)grid > n_stages && !self_clear) grid = (int)n_stages;   // self-clearing: every SM, so launches never overlap
+    p.drop_stage = -1;
+    if (fmt == LW_Q4_0 && nt == 1) {
+        // testing aid: a pending lw_debug_drop_copy request is consumed by this launch
+        const int drop = take_drop_unit();
+        if (drop >= 0) {
+            p.drop_stage = drop;
+            return launch_mma<MmaQ40, 1, true>(p, maps, grid, smem_bytes, overlap != 0, stream);
+        }
+    }
     if (fmt == LW_Q4_0)
         return nt == 1 ? launch_mma<MmaQ40, 1>(p, maps, grid, smem_bytes, overlap != 0, stream)
                        : launch_mma<MmaQ40, 2>(p, maps, grid, smem_bytes, overlap != 0, stream);

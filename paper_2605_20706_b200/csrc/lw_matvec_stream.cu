@@ -582,7 +582,6 @@ std::atomic<int>& drop_unit_storage() {
     static std::atomic<int> v{-1};
     return v;
 }
-int take_drop_unit() { return drop_unit_storage().exchange(-1); }
 
 constexpr size_t kSmemPerSm = 233472;      // 228 KB of shared memory per SM, 1 KB reserved per CTA
 constexpr size_t kSmemMaxCta = 227 * 1024;    // largest opt-in dynamic shared memory of a CTA
@@ -798,6 +797,7 @@ int batched_columns(int fmt, int64_t rows, int64_t cols) {
 }  // namespace
 
 void set_drop_unit(int unit) { drop_unit_storage().store(unit < 0 ? -1 : unit); }
+int take_drop_unit() { return drop_unit_storage().exchange(-1); }
 
 void set_shape_tuning(int fmt, int64_t rows, int64_t cols, int worker_groups, int stages, int stage_kb) {
     std::vector<ShapeTuning>& t = shape_table();

@@ -271,3 +271,34 @@ def test_a_copy_that_never_comes_is_reported_and_the_library_stays_usable():
     y2 = _run(fmt, blocks, rows, cols, X)         # the request was consumed: this call is an ordinary one
     check_matvec(y2, y_ref, s_ref, "call after the fault")
     assert lw.device_status() == 0
+
+
+@pytest.mark.parametrize("overlap", [0, 2])
+def test_a_copy_that_never_comes_in_the_tensor_core_kernel(overlap):
+    # the same aid in the batched tensor-core kernel: from its second stage on a CTA's producer requests nothing, the
+    # compute warps' wait for that stage runs out, the fault is recorded, the CTA stops waiting and the kernel ends;
+    # the next call is an ordinary one.  Both launch forms (self-clearing cooperative launch, clearing kernel chained
+    # by programmatic dependent launch).
+    fmt, rows, cols, batch = lw.Q4_0, 4096, 4096, 8
+    blocks = quantized_weights(fmt, rows, cols, seed=98)
+    X = synth.activations(98, 0, batch, cols)
+    y_ref, s_ref = oracle.matvec(fmt, blocks, rows, cols, X, batch, nthreads=8)
+    assert lw.device_status() == 0
+    w = torch.from_numpy(blocks).cuda()
+    x = torch.from_numpy(X).cuda()
+    y = Guarded((batch, rows))
+    lw.set_variant(lw.VARIANT_AUTO)
+    lw.set_overlap(overlap)
+    try:
+        assert lw.query_variant(fmt, rows, cols, batch) == lw.VARIANT_MMA
+        lw.debug_drop_copy(1)
+        lw.matvec(fmt, w, rows, cols, x, y.t, batch)
+        torch.cuda.synchronize()                  # the kernel ends by itself (one bounded wait of ~0.1 s per warp)
+        y.check("Y of the faulted call")
+        assert lw.device_status() != 0
+        assert lw.device_status() == 0
+        y2 = _run(fmt, blocks, rows, cols, X, lw.VARIANT_AUTO, batch)
+        check_matvec(y2, y_ref, s_ref, "call after the fault")
+        assert lw.device_status() == 0
+    finally:
+        lw.set_overlap(0)
