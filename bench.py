@@ -48,11 +48,14 @@ SINGLE_WORKLOADS = ("q8_0_2048",)
 DEQUANT_WORKLOADS = tuple("dequant_" + f for f in FMT_ID)
 
 
-MMA_FORMATS = ("q8_0", "q4_0", "q4_K", "q5_K")       # formats the batched tensor-core kernel takes
+MMA_FORMATS = ("q8_0", "q4_0", "q4_K", "q5_K", "f16")       # formats the batched tensor-core kernel takes
 
 
 def arithmetic_of(fmt, batch):
     """What the kernels compute in (the `dtype` key): not a precision claim, the arithmetic that runs."""
+    if fmt == "f16" and batch >= 3:
+        return ("f32 in/out; f16 weights x three-term f16 split of the block-scaled fp32 activations on the tensor cores "
+                "(mma m16n8k16), fp32 accumulation")
     if fmt == "f16":
         return "f32 in/out; f16 weights widened, fp32 FMA"
     if batch == 1:

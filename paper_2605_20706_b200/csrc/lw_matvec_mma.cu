@@ -1,4 +1,4 @@
-// Batched mat-vec on the tensor cores (batch 2..16; q4_0, q8_0, q4_K and q5_K) [paper Sec 3.2: from a handful of columns on
+// Batched mat-vec on the tensor cores (batch 2..16; q4_0, q8_0, q4_K, q5_K and f16) [paper Sec 3.2: from a handful of columns on
 // the mat-vec turns into a small mat-mat product, a dense contraction; Sec 3.3: one decode routine per format
 // spliced into a common skeleton].
 //
@@ -131,6 +131,10 @@ __device__ __forceinline__ float lds_half(uint32_t base) {
     return __half2float(__ushort_as_half(h));
 }
 template <int OFF>
+__device__ __forceinline__ void lds64(uint32_t base, uint32_t& a, uint32_t& b) {
+    asm volatile("ld.shared.v2.b32 {%0, %1}, [%2+%3];" : "=r"(a), "=r"(b) : "r"(base), "n"(OFF));
+}
+template <int OFF>
 __device__ __forceinline__ void lds_f32x2(uint32_t base, float& a, float& b) {
     asm volatile("ld.shared.v2.f32 {%0, %1}, [%2+%3];" : "=f"(a), "=f"(b) : "r"(base), "n"(OFF));
 }
@@ -179,6 +183,8 @@ __device__ __forceinline__ uint32_t bytes_to_bf16_128_plus(uint32_t v) {
 // p[2], p[3] = weights 16+4t .. 16+4t+3 (the k order the B fragments follow).  `wt` = shared-memory address of
 // the row's piece of the stage plus 4 t (t = lane % 4), OFF = byte offset of the two-block unit from there.
 struct MmaQ40 {
+    static constexpr int kStageRows = 256;          // 16 warps x 16 rows
+    static constexpr bool kF16 = false;
     static constexpr int kPiece = 8 * 18;               // bytes of a row's 256 columns
     static constexpr bool kHasMin = false;              // no per-block offset term
     static constexpr int kTableBytes = 0;               // no per-warp table of decoded scales
@@ -207,6 +213,8 @@ struct MmaQ40 {
 };
 
 struct MmaQ80 {
+    static constexpr int kStageRows = 256;          // 16 warps x 16 rows
+    static constexpr bool kF16 = false;
     static constexpr int kPiece = 8 * 34;
     static constexpr bool kHasMin = false;
     static constexpr int kTableBytes = 0;
@@ -246,6 +254,8 @@ struct MmaQ80 {
 // is huge beside its neighbours and meets a weight near zero leaves an absolute error (the extra term E of the
 // accuracy statement).  The 6-bit fields are unpacked once per warp and stage into a table of (d * sc, dmin * m).
 struct MmaQ4K {
+    static constexpr int kStageRows = 256;          // 16 warps x 16 rows
+    static constexpr bool kF16 = false;
     static constexpr int kPiece = 144;
     static constexpr bool kHasMin = true;
     static constexpr int kTableBytes = 16 * 8 * 8;      // per warp: 16 rows x 8 sub-blocks x (d * sc, dmin * m)
@@ -298,6 +308,8 @@ struct MmaQ4K {
 // q5_K: q4_K's layout with 32 bytes of fifth bits between the scales and the nibbles (176 bytes per 256 weights): bit
 // s of byte l is the high bit of weight l of sub-block s, so a code is 0..31 -- still exact in bf16.
 struct MmaQ5K {
+    static constexpr int kStageRows = 256;          // 16 warps x 16 rows
+    static constexpr bool kF16 = false;
     static constexpr int kPiece = 176;
     static constexpr bool kHasMin = true;
     static constexpr int kTableBytes = MmaQ4K::kTableBytes;
@@ -345,6 +357,77 @@ struct MmaQ5K {
         lds_f32x2<(ROW / kPiece) * 64 + 8 * (2 * U + BLK)>(tabg, d, m);
     }
 };
+
+// f16 weights: they are the A operand as they lie in memory (mma with f16 operands), nothing is decoded.  A row's
+// 256 columns are 512 bytes, fetched as four 128-byte slices (one per 64-column unit) with the 128-byte swizzle of
+// the tensor copy, so that the eight rows a warp reads at once fall into different banks: 16-byte chunk c of row r
+// of a slice sits at chunk c ^ (r % 8).  A stage is 128 rows; warps 0-7 take units 0 and 1 of their 16 rows, warps
+// 8-15 units 2 and 3.  The activations are held as three f16 terms of x * s, s a power of two per block of 32 and
+// column that brings the block's largest magnitude to 2^14..2^15: terms one and two are cut off exactly, the
+// third rounds what is left (at most 2^-38 of the block's largest magnitude is lost per element: the extra term E
+// of the accuracy statement with a tiny constant); 1 / s multiplies the block's sum.
+struct MmaF16 {
+    static constexpr int kStageRows = 128;
+    static constexpr bool kF16 = true;
+    static constexpr int kPiece = 512;
+    static constexpr bool kHasMin = false;
+    static constexpr int kTableBytes = 0;
+    static constexpr int kSliceBytes = kStageRows * 128;     // one unit of all the stage's rows
+};
+
+__device__ __forceinline__ void mma_f16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                        uint32_t b1) {
+    asm("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+        "{%0, %1, %2, %3};"
+        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void mma_f16_first(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                              uint32_t b0, uint32_t b1) {
+    asm("{\n\t.reg .f32 z;\n\tmov.f32 z, 0f00000000;\n\t"
+        "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0, %1, %2, %3}, {%4, %5, %6, %7}, {%8, %9}, "
+        "{z, z, z, z};\n\t}"
+        : "=f"(d[0]), "=f"(d[1]), "=f"(d[2]), "=f"(d[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+// One block of 32 f16 weights of the warp's 16 rows against all columns.  wrow = address of row g's 128 bytes in
+// slice 0 of the stage plus 8 (t % 2); sw[h] = byte offset of the lane's swizzled 16-byte chunk for half h of block
+// 0 (block 1: sw[2 + h]); sx = the lane's two block scales (1 / s), group nt 32 bytes further.
+template <int NT, int U, int BLK>
+__device__ __forceinline__ void block_step_f16(uint32_t wrow, const uint32_t (&sw)[4], uint32_t sx,
+                                               const uint32_t (&xp)[NT][3], float (&y)[NT][4]) {
+    constexpr int kSlice = U * MmaF16::kSliceBytes;
+    uint32_t a[4], b[4];
+    lds64<kSlice>(wrow + sw[2 * BLK], a[0], a[1]);               // row g: k = 4t .. 4t+3
+    lds64<kSlice>(wrow + sw[2 * BLK + 1], a[2], a[3]);           //        k = 16+4t ..
+    lds64<kSlice + 8 * 128>(wrow + sw[2 * BLK], b[0], b[1]);     // row g + 8 (same swizzle: (g + 8) % 8 == g)
+    lds64<kSlice + 8 * 128>(wrow + sw[2 * BLK + 1], b[2], b[3]);
+    constexpr int kX = 2 * (64 * U + 32 * BLK);
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+        float c[4];
+#pragma unroll
+        for (int s = 0; s < 3; ++s) {
+            uint32_t b0, b1, b2, b3;
+            lds128<kX>(xp[nt][s], b0, b1, b2, b3);
+            if (s == 0)
+                mma_f16_first(c, a[0], b[0], a[1], b[1], b0, b1);
+            else
+                mma_f16(c, a[0], b[0], a[1], b[1], b0, b1);
+            mma_f16(c, a[2], b[2], a[3], b[3], b2, b3);
+        }
+        float s0, s1;                                            // 1 / s of columns 2 t and 2 t + 1 of the group
+        if (nt == 0)
+            lds_f32x2<kSxBlockBytes * (2 * U + BLK)>(sx, s0, s1);
+        else
+            lds_f32x2<kSxBlockBytes * (2 * U + BLK) + 32>(sx, s0, s1);
+        y[nt][0] = fmaf(s0, c[0], y[nt][0]);
+        y[nt][1] = fmaf(s1, c[1], y[nt][1]);
+        y[nt][2] = fmaf(s0, c[2], y[nt][2]);
+        y[nt][3] = fmaf(s1, c[3], y[nt][3]);
+    }
+}
 
 // One block (32 weights) of the warp's 16 rows against all columns: decode the lane's fragments of rows g and
 // g + 8, six products per group of eight columns into one accumulator, then the block scales in fp32.
@@ -406,6 +489,18 @@ __device__ __forceinline__ void split3(float x, uint32_t& h1, uint32_t& h2, uint
     h3 = __float_as_uint(r2) >> 16;                     // at most eight significant bits are left: exact
 }
 
+// fp32 -> three f16 terms of x (already scaled into the f16 range): the first two cut off (exact differences), the
+// third rounds the rest
+__device__ __forceinline__ void split3_f16(float x, uint32_t& h1, uint32_t& h2, uint32_t& h3) {
+    unsigned short a, b, c;
+    asm("cvt.rz.f16.f32 %0, %1;" : "=h"(a) : "f"(x));
+    const float r1 = x - __half2float(__ushort_as_half(a));
+    asm("cvt.rz.f16.f32 %0, %1;" : "=h"(b) : "f"(r1));
+    const float r2 = r1 - __half2float(__ushort_as_half(b));
+    asm("cvt.rn.f16.f32 %0, %1;" : "=h"(c) : "f"(r2));
+    h1 = a, h2 = b, h3 = c;
+}
+
 // Clears Y for the kernel below.  Launched like it (see launch_matvec_mma): lets its successor start its set-up
 // at once and waits for its predecessor before it writes.
 __global__ void __launch_bounds__(256) zero_kernel(float4* __restrict__ y, int64_t quads, float* __restrict__ tail,
@@ -462,6 +557,7 @@ __global__ void __launch_bounds__(kMmaThreads, kCtasPerSm) matvec_mma_kernel(con
     volatile int* stop = reinterpret_cast<volatile int*>(smem + 64);  // set when a wait gave up
     constexpr int NB = 8 * NT;                                        // columns held (beyond the batch: zeros)
     constexpr int kPiece = T::kPiece;                                 // bytes of a row's share of a stage
+    constexpr int kStageRows = T::kStageRows;                         // (shadows the 256 of the quantised formats)
     constexpr int kStageBytes = kStageRows * kPiece;
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
@@ -511,9 +607,18 @@ __global__ void __launch_bounds__(kMmaThreads, kCtasPerSm) matvec_mma_kernel(con
                 break;
             }
             mbar_expect_tx(&full[cur.slot], kStageBytes);   // a box always delivers all its bytes (zeros past the end)
-            tensor_load_2d(smem + p.w_off + (size_t)cur.slot * kStageBytes, &maps.m[cur.it],
-                           (cur.c * spc + cur.j) * (kPiece / 4), (cur.rs - p.item[cur.it].rs_begin) * kStageRows,
-                           &full[cur.slot], policy);
+            if constexpr (T::kF16) {
+                // four swizzled 128-byte slices (one per 64-column unit), each all the stage's rows
+#pragma unroll
+                for (int u = 0; u < 4; ++u)
+                    tensor_load_2d(smem + p.w_off + (size_t)cur.slot * kStageBytes + u * MmaF16::kSliceBytes,
+                                   &maps.m[cur.it], ((cur.c * spc + cur.j) * 4 + u) * 32,
+                                   (cur.rs - p.item[cur.it].rs_begin) * kStageRows, &full[cur.slot], policy);
+            } else {
+                tensor_load_2d(smem + p.w_off + (size_t)cur.slot * kStageBytes, &maps.m[cur.it],
+                               (cur.c * spc + cur.j) * (kPiece / 4), (cur.rs - p.item[cur.it].rs_begin) * kStageRows,
+                               &full[cur.slot], policy);
+            }
         }
         if (*stop) {
             // the consumers have stopped waiting: make sure nothing is still landing in shared memory (stage m,
@@ -556,7 +661,13 @@ __global__ void __launch_bounds__(kMmaThreads, kCtasPerSm) matvec_mma_kernel(con
     const uint32_t xs = smem_u32(smem + p.x_off);
     // this lane's B fragments: column g of each group of eight, slots 8 t .. 8 t + 7 of a block of 32
     const uint32_t xlane = xs + g * x_pitch + 16u * t;
-    const uint32_t wrow = smem_u32(smem + p.w_off) + (uint32_t)(16 * warp + g) * kPiece;   // row g of this warp's 16
+    // the warp's 16 rows of a stage; f16: 128-row stages, warps 0-7 take units 0 and 1, warps 8-15 units 2 and 3
+    const int mt = T::kF16 ? (warp & 7) : warp;
+    const uint32_t wrow = smem_u32(smem + p.w_off) +
+                          (T::kF16 ? (uint32_t)(16 * mt + g) * 128u + 8u * (t & 1) : (uint32_t)(16 * warp + g) * kPiece);
+    uint32_t sw[4];                                     // f16: the lane's swizzled chunk offsets (see block_step_f16)
+#pragma unroll
+    for (int i = 0; i < 4; ++i) sw[i] = (uint32_t)(((2 * i + (t >> 1)) ^ g) << 4);
 
     float y[NT][4];
 #pragma unroll
@@ -585,7 +696,7 @@ __global__ void __launch_bounds__(kMmaThreads, kCtasPerSm) matvec_mma_kernel(con
             cleared = true;
         }
         const MmaItem& m = p.item[cur_it];
-        const int64_t r = (int64_t)(cur_rs - m.rs_begin) * kStageRows + 16 * warp + g;
+        const int64_t r = (int64_t)(cur_rs - m.rs_begin) * kStageRows + 16 * mt + g;
 #pragma unroll
         for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
@@ -643,10 +754,29 @@ __global__ void __launch_bounds__(kMmaThreads, kCtasPerSm) matvec_mma_kernel(con
                         const int idx = tid + nt * kMmaComputeThreads;
                         const int b = idx >> 6, k4 = jj * (kStageCols / 4) + (idx & 63);
                         uint32_t h[3][4];
-                        split3(v[q][nt].x, h[0][0], h[1][0], h[2][0]);
-                        split3(v[q][nt].y, h[0][1], h[1][1], h[2][1]);
-                        split3(v[q][nt].z, h[0][2], h[1][2], h[2][2]);
-                        split3(v[q][nt].w, h[0][3], h[1][3], h[2][3]);
+                        if constexpr (T::kF16) {
+                            // f16 terms of x * s, s = the power of two that brings the block's largest magnitude (eight
+                            // consecutive lanes hold a block of 32) to 2^14 .. 2^15; 1 / s goes to [block][column]
+                            float mx = fmaxf(fmaxf(fabsf(v[q][nt].x), fabsf(v[q][nt].y)), fmaxf(fabsf(v[q][nt].z), fabsf(v[q][nt].w)));
+                            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
+                            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 2));
+                            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
+                            int se = 268 - (int)((__float_as_uint(mx) >> 23) & 0xFFu);      // biased exponent of s
+                            se = se < 1 ? 1 : (se > 253 ? 253 : se);
+                            const float sc = __uint_as_float((uint32_t)se << 23);
+                            if ((lane & 7) == 0)
+                                *reinterpret_cast<float*>(smem + p.sx_off + (size_t)(k4 >> 3) * kSxBlockBytes + 4 * b) =
+                                    __uint_as_float((uint32_t)(254 - se) << 23);
+                            split3_f16(v[q][nt].x * sc, h[0][0], h[1][0], h[2][0]);
+                            split3_f16(v[q][nt].y * sc, h[0][1], h[1][1], h[2][1]);
+                            split3_f16(v[q][nt].z * sc, h[0][2], h[1][2], h[2][2]);
+                            split3_f16(v[q][nt].w * sc, h[0][3], h[1][3], h[2][3]);
+                        } else {
+                            split3(v[q][nt].x, h[0][0], h[1][0], h[2][0]);
+                            split3(v[q][nt].y, h[0][1], h[1][1], h[2][1]);
+                            split3(v[q][nt].z, h[0][2], h[1][2], h[2][2]);
+                            split3(v[q][nt].w, h[0][3], h[1][3], h[2][3]);
+                        }
                         if constexpr (T::kHasMin) {
                             // sum of each block of 32 activations (eight consecutive lanes hold one), for the
                             // formats with a per-block offset: [block of the chunk][column]
@@ -676,7 +806,7 @@ __global__ void __launch_bounds__(kMmaThreads, kCtasPerSm) matvec_mma_kernel(con
             }
         }
         const int64_t r0 = (int64_t)(rs - mat.rs_begin) * kStageRows;
-        if (r0 + 16 * warp < mat.rows) {
+        if (r0 + 16 * mt < mat.rows) {
             const uint32_t row = wrow + (uint32_t)slot * kStageBytes, wt = row + 4u * t;
             const uint32_t tab = smem_u32(smem + p.tab_off) + (uint32_t)warp * T::kTableBytes, tabg = tab + 64u * g;
             const uint32_t sx = smem_u32(smem + p.sx_off) + (uint32_t)(8 * j) * kSxBlockBytes + 8u * t;
@@ -690,14 +820,29 @@ __global__ void __launch_bounds__(kMmaThreads, kCtasPerSm) matvec_mma_kernel(con
 #pragma unroll
                 for (int s = 0; s < 3; ++s)
                     xp[nt][s] = xlane + 2u * (uint32_t)(j * kStageCols) + s * plane_pitch + nt * 8 * x_pitch;
-            block_step<T, NT, 0, 0>(wt, row, tabg, sx, xp, y);
-            block_step<T, NT, 0, 1>(wt, row, tabg, sx, xp, y);
-            block_step<T, NT, 1, 0>(wt, row, tabg, sx, xp, y);
-            block_step<T, NT, 1, 1>(wt, row, tabg, sx, xp, y);
-            block_step<T, NT, 2, 0>(wt, row, tabg, sx, xp, y);
-            block_step<T, NT, 2, 1>(wt, row, tabg, sx, xp, y);
-            block_step<T, NT, 3, 0>(wt, row, tabg, sx, xp, y);
-            block_step<T, NT, 3, 1>(wt, row, tabg, sx, xp, y);
+            if constexpr (T::kF16) {
+                const uint32_t wr = wrow + (uint32_t)slot * kStageBytes;
+                if (warp < 8) {
+                    block_step_f16<NT, 0, 0>(wr, sw, sx, xp, y);
+                    block_step_f16<NT, 0, 1>(wr, sw, sx, xp, y);
+                    block_step_f16<NT, 1, 0>(wr, sw, sx, xp, y);
+                    block_step_f16<NT, 1, 1>(wr, sw, sx, xp, y);
+                } else {
+                    block_step_f16<NT, 2, 0>(wr, sw, sx, xp, y);
+                    block_step_f16<NT, 2, 1>(wr, sw, sx, xp, y);
+                    block_step_f16<NT, 3, 0>(wr, sw, sx, xp, y);
+                    block_step_f16<NT, 3, 1>(wr, sw, sx, xp, y);
+                }
+            } else {
+                block_step<T, NT, 0, 0>(wt, row, tabg, sx, xp, y);
+                block_step<T, NT, 0, 1>(wt, row, tabg, sx, xp, y);
+                block_step<T, NT, 1, 0>(wt, row, tabg, sx, xp, y);
+                block_step<T, NT, 1, 1>(wt, row, tabg, sx, xp, y);
+                block_step<T, NT, 2, 0>(wt, row, tabg, sx, xp, y);
+                block_step<T, NT, 2, 1>(wt, row, tabg, sx, xp, y);
+                block_step<T, NT, 3, 0>(wt, row, tabg, sx, xp, y);
+                block_step<T, NT, 3, 1>(wt, row, tabg, sx, xp, y);
+            }
         }
         __syncwarp();
         if (lane == 0) mbar_arrive(&empty[slot]);
@@ -752,17 +897,21 @@ EncodeTiledFn encode_tiled_fn() {
     return fn;
 }
 
-// The weight matrix as a 2-D tensor of 32-bit words (row_bytes / 4 per row, `rows` rows) with boxes of one stage.
-bool make_weight_map(CUtensorMap* map, const void* W, int64_t rows, int64_t row_bytes, int piece_bytes) {
+int mma_stage_rows(int fmt) { return fmt == LW_F16 ? MmaF16::kStageRows : kStageRows; }
+
+// The weight matrix as a 2-D tensor of 32-bit words (row_bytes / 4 per row, `rows` rows) with boxes of one stage;
+// f16: boxes of one 128-byte slice of a stage's rows, written with the 128-byte swizzle.
+bool make_weight_map(CUtensorMap* map, int fmt, const void* W, int64_t rows, int64_t row_bytes, int piece_bytes) {
     EncodeTiledFn fn = encode_tiled_fn();
     if (!fn) return false;
+    const bool f16 = fmt == LW_F16;
     const cuuint64_t dims[2] = {(cuuint64_t)(row_bytes / 4), (cuuint64_t)rows};
     const cuuint64_t strides[1] = {(cuuint64_t)row_bytes};
-    const cuuint32_t box[2] = {(cuuint32_t)(piece_bytes / 4), (cuuint32_t)kStageRows};
+    const cuuint32_t box[2] = {(cuuint32_t)(f16 ? 32 : piece_bytes / 4), (cuuint32_t)mma_stage_rows(fmt)};
     const cuuint32_t elem[2] = {1, 1};
     return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<void*>(W), dims, strides, box, elem,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+              CU_TENSOR_MAP_INTERLEAVE_NONE, f16 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+              CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 int mma_sm_count() {
@@ -776,13 +925,18 @@ int mma_sm_count() {
 // for at least two stages.  Returns false if nothing fits.
 bool mma_plan(int fmt, int64_t cols, int nt, int& chunk_cols, int& ring, size_t& x_bytes, size_t& stage_bytes,
               size_t& extra_bytes) {
-    const int piece = fmt == LW_Q8_0 ? MmaQ80::kPiece
-                                     : fmt == LW_Q4_0 ? MmaQ40::kPiece : fmt == LW_Q4_K ? MmaQ4K::kPiece : MmaQ5K::kPiece;
-    stage_bytes = (size_t)kStageRows * piece;
+    const int piece = fmt == LW_Q8_0   ? MmaQ80::kPiece
+                      : fmt == LW_Q4_0 ? MmaQ40::kPiece
+                      : fmt == LW_Q4_K ? MmaQ4K::kPiece
+                      : fmt == LW_Q5_K ? MmaQ5K::kPiece
+                                       : MmaF16::kPiece;
+    stage_bytes = (size_t)mma_stage_rows(fmt) * piece;
     // q4_K: block sums of the activations (64 bytes per block of a chunk of up to 1024 columns) and the warps' tables
     extra_bytes = (fmt == LW_Q4_K || fmt == LW_Q5_K)
-                      ? (size_t)(1024 / 32) * kSxBlockBytes + (size_t)kMmaWarps * MmaQ4K::kTableBytes : 0;
-    const size_t budget = kSmemPerCta - kMmaHeader - extra_bytes;
+                      ? (size_t)(1024 / 32) * kSxBlockBytes + (size_t)kMmaWarps * MmaQ4K::kTableBytes
+                      : (fmt == LW_F16 ? (size_t)(1024 / 32) * kSxBlockBytes : 0);
+    // (f16: up to 1 KB more goes into aligning the swizzled stages)
+    const size_t budget = kSmemPerCta - kMmaHeader - extra_bytes - (fmt == LW_F16 ? 1024 : 0);
     // the largest chunk that leaves room for two stages (q8_0, 458752 x 4096, 8 columns: 0.40 ms with chunks of
     // 1024 columns and two 68 KB stages against 0.49 ms with chunks of 256 and three)
     for (int kx = 1024; kx >= 256; kx /= 2) {
@@ -800,7 +954,7 @@ bool mma_plan(int fmt, int64_t cols, int nt, int& chunk_cols, int& ring, size_t&
 }  // namespace
 
 bool matvec_mma_supported(int fmt, int64_t rows, int64_t cols, int batch) {
-    if (fmt != LW_Q4_0 && fmt != LW_Q8_0 && fmt != LW_Q4_K && fmt != LW_Q5_K) return false;
+    if (fmt != LW_Q4_0 && fmt != LW_Q8_0 && fmt != LW_Q4_K && fmt != LW_Q5_K && fmt != LW_F16) return false;
     if (batch < 2 || batch > 16) return false;
     if (cols % kStageCols != 0) return false;
     return rows >= 1 && rows <= (int64_t)1 << 30;
@@ -811,7 +965,7 @@ bool matvec_mma_group_supported(int fmt, int64_t cols, int n_items, const int64_
     int64_t total_rs = 0;
     for (int i = 0; i < n_items; ++i) {
         if (!matvec_mma_supported(fmt, rows[i], cols, batch)) return false;
-        total_rs += (rows[i] + kStageRows - 1) / kStageRows;
+        total_rs += (rows[i] + mma_stage_rows(fmt) - 1) / mma_stage_rows(fmt);
     }
     return total_rs * (cols / kStageCols) < ((int64_t)1 << 31);
 }
@@ -835,7 +989,7 @@ int launch_matvec_mma_group(int fmt, int64_t cols, int n_items, const void* cons
         int cc = 0, rg = 0;
         size_t xb = 0, sb = 0, eb = 0;
         if (!mma_plan(fmt, cols, batch > 8 ? 2 : 1, cc, rg, xb, sb, eb)) return (int)cudaErrorInvalidValue;
-        if (2 * ((kMmaHeader + xb + eb + 127) / 128 * 128 + (size_t)rg * sb + 1024) <= 228 * 1024 || kCtasPerSm != 1)
+        if (2 * ((kMmaHeader + xb + eb + 127) / 128 * 128 + (size_t)rg * sb + 1024) <= 228 * 1024 || kCtasPerSm != 1)   // (f16's alignment slack only adds)
             self_clear = false;
     }
     unsigned* grid_bar = nullptr;
@@ -872,8 +1026,8 @@ int launch_matvec_mma_group(int fmt, int64_t cols, int n_items, const void* cons
         p.item[i].Y = Y[i];
         p.item[i].rows = rows[i];
         p.item[i].rs_begin = rs;
-        rs += (int)((rows[i] + kStageRows - 1) / kStageRows);
-        if (!make_weight_map(&maps.m[i], W[i], rows[i], row_bytes, (int)(stage_bytes / kStageRows)))
+        rs += (int)((rows[i] + mma_stage_rows(fmt) - 1) / mma_stage_rows(fmt));
+        if (!make_weight_map(&maps.m[i], fmt, W[i], rows[i], row_bytes, (int)(stage_bytes / mma_stage_rows(fmt))))
             return (int)cudaErrorInvalidValue;
     }
     for (int i = n_items - 1; i >= 0; --i)          // end of the run of matrices that read the same X
@@ -890,7 +1044,9 @@ int launch_matvec_mma_group(int fmt, int64_t cols, int n_items, const void* cons
     p.x_off = kMmaHeader;
     p.sx_off = (uint32_t)(kMmaHeader + x_bytes);
     p.tab_off = p.sx_off + (uint32_t)((fmt == LW_Q4_K || fmt == LW_Q5_K) ? (1024 / 32) * kSxBlockBytes : 0);
-    p.w_off = (uint32_t)((kMmaHeader + x_bytes + extra_bytes + 127) / 128 * 128);
+    // the stages: 128-byte aligned; f16's swizzle pattern is one of address bits, so its stages start on 1 KB
+    const size_t w_align = fmt == LW_F16 ? 1024 : 128;
+    p.w_off = (uint32_t)((kMmaHeader + x_bytes + extra_bytes + w_align - 1) / w_align * w_align);
     const size_t smem_bytes = p.w_off + (size_t)p.ring * stage_bytes;
     const int64_t n_stages = (cols / kStageCols) * (int64_t)rs;
     int grid = kCtasPerSm * mma_sm_count();
@@ -913,6 +1069,9 @@ int launch_matvec_mma_group(int fmt, int64_t cols, int n_items, const void* cons
     if (fmt == LW_Q5_K)
         return nt == 1 ? launch_mma<MmaQ5K, 1>(p, maps, grid, smem_bytes, overlap != 0, stream)
                        : launch_mma<MmaQ5K, 2>(p, maps, grid, smem_bytes, overlap != 0, stream);
+    if (fmt == LW_F16)
+        return nt == 1 ? launch_mma<MmaF16, 1>(p, maps, grid, smem_bytes, overlap != 0, stream)
+                       : launch_mma<MmaF16, 2>(p, maps, grid, smem_bytes, overlap != 0, stream);
     return nt == 1 ? launch_mma<MmaQ80, 1>(p, maps, grid, smem_bytes, overlap != 0, stream)
                    : launch_mma<MmaQ80, 2>(p, maps, grid, smem_bytes, overlap != 0, stream);
 }

@@ -131,12 +131,13 @@ def test_batched_kernels_need_no_extra_term(fmt, kernel):
     assert (np.abs(y.astype(np.float64) - y_ref)[finite] <= (RTOL * s_ref + ATOL)[finite]).all()
 
 
-@pytest.mark.parametrize("fmt", [lw.Q4_K, lw.Q5_K])
-def test_k_quants_on_the_tensor_cores_stay_inside_the_stated_bound(fmt):
+@pytest.mark.parametrize("fmt,c_extra", [(lw.Q4_K, 2.0 ** -18), (lw.Q5_K, 2.0 ** -18), (lw.F16, 2.0 ** -30)])
+def test_formats_with_an_extra_term_on_the_tensor_cores_stay_inside_the_stated_bound(fmt, c_extra):
     # q4_K / q5_K in the batched tensor-core kernel apply the sub-block offsets to sums of activations, like the
-    # fp32-activation streaming family: the header gives them the extra term with c = 2^-18, asserted here on the
-    # adversarial activations (eight columns, each with its own outliers), and a non-finite activation stays in its
-    # column
+    # fp32-activation streaming family: the header gives them the extra term with c = 2^-18; f16 holds the
+    # activations as three f16 terms relative to each block's largest magnitude, which can lose up to 2^-38 of that
+    # magnitude per element (c = 2^-30 stated).  Asserted here on the adversarial activations (eight columns, each
+    # with its own outliers); a non-finite activation stays in its column
     rows, cols, batch = 48, 4096, 8
     cols_x = []
     for b in range(batch):
@@ -148,7 +149,7 @@ def test_k_quants_on_the_tensor_cores_stay_inside_the_stated_bound(fmt):
     assert lw.query_variant(fmt, rows, cols, batch) == lw.VARIANT_MMA
     y = _run(fmt, blocks, rows, cols, X, lw.VARIANT_MMA, batch)
     for b in range(batch):
-        bound = RTOL * s_ref[b] + ATOL + _extra_term(fmt, blocks, rows, cols, X[b:b + 1], 2.0 ** -18)[0]
+        bound = RTOL * s_ref[b] + ATOL + _extra_term(fmt, blocks, rows, cols, X[b:b + 1], c_extra)[0]
         worst = float((np.abs(y[b].astype(np.float64) - y_ref[b]) / bound).max())
         assert worst <= 1.0, "column %d: error / bound = %.3g" % (b, worst)
     Xb = X.copy()
