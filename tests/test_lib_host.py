@@ -158,7 +158,8 @@ def test_variant_controls():
         assert lw.query_variant(f, 16, 96, 1) == lw.VARIANT_GENERIC
     assert lw.query_variant(lw.Q6_K, 64, 1024, 1) == lw.VARIANT_GENERIC     # q6_K rows must be whole 16-byte pieces
     assert lw.query_variant(lw.F16, 4096, 4096, 2) == lw.VARIANT_STREAM      # f16, up to 4 columns: one pass per column
-    assert lw.query_variant(lw.F16, 4096, 4096, 8) == lw.VARIANT_GENERIC     # f16, more columns: tiled fp32 kernel
+    assert lw.query_variant(lw.F16, 4096, 4096, 8) == lw.VARIANT_MMA         # f16 from three columns: tensor-core kernel
+    assert lw.query_variant(lw.F16, 4096, 4096 + 128, 8) == lw.VARIANT_GENERIC  # cols % 256 != 0: tiled fp32 kernel
     assert lw.query_variant(lw.Q8_0, 64, 32768, 1) == lw.VARIANT_GENERIC     # too wide for one CTA
     lw.set_variant(lw.VARIANT_STREAM)
     assert lw.query_variant(lw.Q4_0, 4096, 4096, 1) == lw.VARIANT_STREAM
