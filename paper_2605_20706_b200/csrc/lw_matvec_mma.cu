@@ -1,4 +1,4 @@
-// Batched mat-vec on the tensor cores (batch 2..16; q4_0, q8_0, q4_K, q5_K and f16) [paper Sec 3.2: from a handful of columns on
+// Batched mat-vec on the tensor cores (batch 2..16; q4_0, q8_0, q4_K, q5_K, q4_1, q5_0, q5_1 and f16) [paper Sec 3.2: from a handful of columns on
 // the mat-vec turns into a small mat-mat product, a dense contraction; Sec 3.3: one decode routine per format
 // spliced into a common skeleton].
 //
@@ -190,7 +190,7 @@ struct MmaQ40 {
     static constexpr int kTableBytes = 0;               // no per-warp table of decoded scales
     static __device__ __forceinline__ void prepare(uint32_t, uint32_t, int) {}
     template <int U, int BLK, int ROW>
-    static __device__ __forceinline__ void block(uint32_t wt, uint32_t (&p)[4]) {
+    static __device__ __forceinline__ void block(uint32_t wt, uint32_t, int, uint32_t (&p)[4]) {
         constexpr int OFF = ROW + 36 * U;               // the two-block unit
         uint32_t q;
         if (BLK == 0)                                   // quants at bytes 2..17: word t straddles two words
@@ -225,7 +225,7 @@ struct MmaQ80 {
         return sub_bf16x2(v & 0xFF7FFF7Fu, v & 0xFF80FF80u);
     }
     template <int U, int BLK, int ROW>
-    static __device__ __forceinline__ void block(uint32_t wt, uint32_t (&p)[4]) {
+    static __device__ __forceinline__ void block(uint32_t wt, uint32_t, int, uint32_t (&p)[4]) {
         constexpr int OFF = ROW + 68 * U;
         uint32_t qa, qb;                                // quant words t and 4 + t of the block
         if (BLK == 0) {                                 // quants at bytes 2..33
@@ -283,7 +283,7 @@ struct MmaQ4K {
         }
     }
     template <int U, int BLK, int ROW>
-    static __device__ __forceinline__ void block(uint32_t wt, uint32_t (&p)[4]) {
+    static __device__ __forceinline__ void block(uint32_t wt, uint32_t, int, uint32_t (&p)[4]) {
         constexpr int OFF = ROW + 16 + 32 * U;          // the 32 bytes of sub-blocks 2 U (low nibbles), 2 U + 1 (high)
         uint32_t qa = lds32<OFF>(wt), qb = lds32<OFF + 16>(wt);         // bytes 4t .. 4t+3 and 16+4t .. 16+4t+3
         if (BLK == 1) {
@@ -336,7 +336,7 @@ struct MmaQ5K {
         }
     }
     template <int U, int BLK, int ROW>
-    static __device__ __forceinline__ void block(uint32_t wt, uint32_t (&p)[4]) {
+    static __device__ __forceinline__ void block(uint32_t wt, uint32_t, int, uint32_t (&p)[4]) {
         constexpr int S = 2 * U + BLK;                  // sub-block = bit of the fifth-bit bytes
         uint32_t qa = lds32<ROW + 48 + 32 * U>(wt), qb = lds32<ROW + 48 + 32 * U + 16>(wt);
         const uint32_t ha = lds32<ROW + 16>(wt), hb = lds32<ROW + 32>(wt);   // fifth bits of weights 4t.. and 16+4t..
@@ -355,6 +355,62 @@ struct MmaQ5K {
     template <int U, int BLK, int ROW>
     static __device__ __forceinline__ void scales(uint32_t, uint32_t tabg, float& d, float& m) {
         lds_f32x2<(ROW / kPiece) * 64 + 8 * (2 * U + BLK)>(tabg, d, m);
+    }
+};
+
+// Four bits (0..3 of `x`) spread to bit 4 of four bytes: the fifth bits of four 5-bit codes.
+__device__ __forceinline__ uint32_t fifth_bits(uint32_t x) { return ((x & 0xFu) * 0x02040810u) & 0x10101010u; }
+
+// The 32-weight formats with an offset and / or a fifth bit: q4_1 {d, m, 16 bytes of nibbles} = d * q + m, q5_0 {d, 32
+// fifth bits, nibbles} = d * (q - 16), q5_1 {d, m, fifth bits, nibbles} = d * q + m; nibble and bit order as in q4_0
+// (byte j: weights j and j + 16; bit j: weight j).  Codes 0..31 are exact in bf16.  q5_0 has no offset: E = 0; the
+// offsets m of q4_1 / q5_1 go onto fp32 block sums of the activations (extra term E, c = 2^-18).
+template <int FMT>
+struct MmaLegacy {
+    static constexpr bool kFive = FMT != LW_Q4_1;
+    static constexpr bool kHasMin = FMT != LW_Q5_0;
+    static constexpr int kBlock = FMT == LW_Q4_1 ? 20 : (FMT == LW_Q5_0 ? 22 : 24);
+    static constexpr int kStageRows = 256;
+    static constexpr bool kF16 = false;
+    static constexpr int kPiece = 8 * kBlock;
+    static constexpr int kTableBytes = 0;
+    static __device__ __forceinline__ void prepare(uint32_t, uint32_t, int) {}
+    // wt = the row's piece + 4 t, row = the row's piece, t = lane % 4
+    template <int U, int BLK, int ROW>
+    static __device__ __forceinline__ void block(uint32_t wt, uint32_t row, int t, uint32_t (&p)[4]) {
+        constexpr int B0 = ROW + 2 * kBlock * U + kBlock * BLK;       // the block, in bytes from the row's piece
+        uint32_t q, qh = 0;
+        if constexpr (FMT == LW_Q4_1) {
+            q = lds32<B0 + 4>(wt);
+        } else if constexpr (FMT == LW_Q5_1) {
+            q = lds32<B0 + 8>(wt);
+            qh = lds32<B0 + 4>(row);
+        } else if constexpr (BLK == 0) {                             // q5_0, block at 44 U: fields two bytes off a word
+            q = __byte_perm(lds32<B0 + 4>(wt), lds32<B0 + 8>(wt), 0x5432u);         // nibble bytes 6 + 4t ..
+            qh = __byte_perm(lds32<B0>(row), lds32<B0 + 4>(row), 0x5432u);          // fifth bits at bytes 2 .. 5
+        } else {                                                     // q5_0, block at 44 U + 22: fields on words
+            q = lds32<B0 + 6>(wt);
+            qh = lds32<B0 + 2>(row);
+        }
+        uint32_t lo = q & 0x0F0F0F0Fu, hi = (q >> 4) & 0x0F0F0F0Fu;
+        if constexpr (kFive) {
+            const uint32_t h = qh >> (4 * t);                        // bits 4t .. 4t+3: weights 4t ..; 16 higher: 16+4t ..
+            lo |= fifth_bits(h);
+            hi |= fifth_bits(h >> 16);
+        }
+        const uint32_t bias = FMT == LW_Q5_0 ? 0x43104310u : 0x43004300u;     // (128 + q) - 144 = q - 16, resp. - 128 = q
+        p[0] = sub_bf16x2(bytes_to_bf16_128_plus<0>(lo), bias);
+        p[1] = sub_bf16x2(bytes_to_bf16_128_plus<2>(lo), bias);
+        p[2] = sub_bf16x2(bytes_to_bf16_128_plus<0>(hi), bias);
+        p[3] = sub_bf16x2(bytes_to_bf16_128_plus<2>(hi), bias);
+    }
+    // (d, minus the offset: the caller subtracts m times the block's sum of activations)
+    template <int U, int BLK, int ROW>
+    static __device__ __forceinline__ void scales(uint32_t row, uint32_t, float& d, float& m) {
+        constexpr int B0 = ROW + 2 * kBlock * U + kBlock * BLK;
+        d = lds_half<B0>(row);
+        if constexpr (kHasMin) m = -lds_half<B0 + 2>(row);
+        else m = 0.f;
     }
 };
 
@@ -440,8 +496,9 @@ __device__ __forceinline__ void block_step(uint32_t wt, uint32_t row, uint32_t t
                                            const uint32_t (&xp)[NT][3], float (&y)[NT][4]) {
     constexpr int kPiece = T::kPiece;
     uint32_t a[4], b[4];
-    T::template block<U, BLK, 0>(wt, a);
-    T::template block<U, BLK, 8 * kPiece>(wt, b);
+    const int t = (int)((wt - row) >> 2);
+    T::template block<U, BLK, 0>(wt, row, t, a);
+    T::template block<U, BLK, 8 * kPiece>(wt, row, t, b);
     float d0, d1, m0, m1;
     T::template scales<U, BLK, 0>(row, tabg, d0, m0);
     T::template scales<U, BLK, 8 * kPiece>(row, tabg, d1, m1);
@@ -929,12 +986,15 @@ bool mma_plan(int fmt, int64_t cols, int nt, int& chunk_cols, int& ring, size_t&
                       : fmt == LW_Q4_0 ? MmaQ40::kPiece
                       : fmt == LW_Q4_K ? MmaQ4K::kPiece
                       : fmt == LW_Q5_K ? MmaQ5K::kPiece
+                      : fmt == LW_Q4_1 ? MmaLegacy<LW_Q4_1>::kPiece
+                      : fmt == LW_Q5_0 ? MmaLegacy<LW_Q5_0>::kPiece
+                      : fmt == LW_Q5_1 ? MmaLegacy<LW_Q5_1>::kPiece
                                        : MmaF16::kPiece;
     stage_bytes = (size_t)mma_stage_rows(fmt) * piece;
     // q4_K: block sums of the activations (64 bytes per block of a chunk of up to 1024 columns) and the warps' tables
     extra_bytes = (fmt == LW_Q4_K || fmt == LW_Q5_K)
                       ? (size_t)(1024 / 32) * kSxBlockBytes + (size_t)kMmaWarps * MmaQ4K::kTableBytes
-                      : (fmt == LW_F16 ? (size_t)(1024 / 32) * kSxBlockBytes : 0);
+                      : ((fmt == LW_F16 || fmt == LW_Q4_1 || fmt == LW_Q5_1) ? (size_t)(1024 / 32) * kSxBlockBytes : 0);
     // (f16: up to 1 KB more goes into aligning the swizzled stages)
     const size_t budget = kSmemPerCta - kMmaHeader - extra_bytes - (fmt == LW_F16 ? 1024 : 0);
     // the largest chunk that leaves room for two stages (q8_0, 458752 x 4096, 8 columns: 0.40 ms with chunks of
@@ -954,7 +1014,9 @@ bool mma_plan(int fmt, int64_t cols, int nt, int& chunk_cols, int& ring, size_t&
 }  // namespace
 
 bool matvec_mma_supported(int fmt, int64_t rows, int64_t cols, int batch) {
-    if (fmt != LW_Q4_0 && fmt != LW_Q8_0 && fmt != LW_Q4_K && fmt != LW_Q5_K && fmt != LW_F16) return false;
+    if (fmt != LW_Q4_0 && fmt != LW_Q8_0 && fmt != LW_Q4_K && fmt != LW_Q5_K && fmt != LW_F16 && fmt != LW_Q4_1 &&
+        fmt != LW_Q5_0 && fmt != LW_Q5_1)
+        return false;
     if (batch < 2 || batch > 16) return false;
     if (cols % kStageCols != 0) return false;
     return rows >= 1 && rows <= (int64_t)1 << 30;
@@ -1072,6 +1134,15 @@ int launch_matvec_mma_group(int fmt, int64_t cols, int n_items, const void* cons
     if (fmt == LW_F16)
         return nt == 1 ? launch_mma<MmaF16, 1>(p, maps, grid, smem_bytes, overlap != 0, stream)
                        : launch_mma<MmaF16, 2>(p, maps, grid, smem_bytes, overlap != 0, stream);
+    if (fmt == LW_Q4_1)
+        return nt == 1 ? launch_mma<MmaLegacy<LW_Q4_1>, 1>(p, maps, grid, smem_bytes, overlap != 0, stream)
+                       : launch_mma<MmaLegacy<LW_Q4_1>, 2>(p, maps, grid, smem_bytes, overlap != 0, stream);
+    if (fmt == LW_Q5_0)
+        return nt == 1 ? launch_mma<MmaLegacy<LW_Q5_0>, 1>(p, maps, grid, smem_bytes, overlap != 0, stream)
+                       : launch_mma<MmaLegacy<LW_Q5_0>, 2>(p, maps, grid, smem_bytes, overlap != 0, stream);
+    if (fmt == LW_Q5_1)
+        return nt == 1 ? launch_mma<MmaLegacy<LW_Q5_1>, 1>(p, maps, grid, smem_bytes, overlap != 0, stream)
+                       : launch_mma<MmaLegacy<LW_Q5_1>, 2>(p, maps, grid, smem_bytes, overlap != 0, stream);
     return nt == 1 ? launch_mma<MmaQ80, 1>(p, maps, grid, smem_bytes, overlap != 0, stream)
                    : launch_mma<MmaQ80, 2>(p, maps, grid, smem_bytes, overlap != 0, stream);
 }

@@ -94,8 +94,8 @@ def test_outliers_on_zero_weights_stay_inside_the_stated_bound(fmt, variant, zer
     assert worst <= 1.0, "variant %d launched %d: error / bound = %.3g" % (variant, launched, worst)
 
 
-@pytest.mark.parametrize("kernel", [lw.VARIANT_TILE, lw.VARIANT_MMA])
-@pytest.mark.parametrize("fmt", [lw.Q8_0, lw.Q4_0])
+@pytest.mark.parametrize("fmt,kernel", [(lw.Q8_0, lw.VARIANT_TILE), (lw.Q4_0, lw.VARIANT_TILE), (lw.Q8_0, lw.VARIANT_MMA),
+                                        (lw.Q4_0, lw.VARIANT_MMA), (lw.Q5_0, lw.VARIANT_MMA)])
 def test_batched_kernels_need_no_extra_term(fmt, kernel):
     # the batched fp32 tile kernel decodes every weight exactly before it multiplies, and the tensor-core kernel
     # multiplies exact integer codes with three bf16 terms that add up to the activation exactly: the plain
@@ -131,7 +131,8 @@ def test_batched_kernels_need_no_extra_term(fmt, kernel):
     assert (np.abs(y.astype(np.float64) - y_ref)[finite] <= (RTOL * s_ref + ATOL)[finite]).all()
 
 
-@pytest.mark.parametrize("fmt,c_extra", [(lw.Q4_K, 2.0 ** -18), (lw.Q5_K, 2.0 ** -18), (lw.F16, 2.0 ** -30)])
+@pytest.mark.parametrize("fmt,c_extra", [(lw.Q4_K, 2.0 ** -18), (lw.Q5_K, 2.0 ** -18), (lw.F16, 2.0 ** -30),
+                                         (lw.Q4_1, 2.0 ** -18), (lw.Q5_1, 2.0 ** -18)])
 def test_formats_with_an_extra_term_on_the_tensor_cores_stay_inside_the_stated_bound(fmt, c_extra):
     # q4_K / q5_K in the batched tensor-core kernel apply the sub-block offsets to sums of activations, like the
     # fp32-activation streaming family: the header gives them the extra term with c = 2^-18; f16 holds the

@@ -79,12 +79,12 @@ def test_matvec_tile_kernel(fmt, batch, rows, cols):
     check_matvec(y, y_ref, s_ref, "tile fmt %d %dx%d batch %d" % (fmt, rows, cols, batch))
 
 
-@pytest.mark.parametrize("fmt", [lw.Q8_0, lw.Q4_0, lw.Q4_K, lw.Q5_K, lw.F16])
+@pytest.mark.parametrize("fmt", [lw.Q8_0, lw.Q4_0, lw.Q4_K, lw.Q5_K, lw.F16, lw.Q4_1, lw.Q5_0, lw.Q5_1])
 @pytest.mark.parametrize("batch", [2, 3, 7, 8, 9, 16])
 @pytest.mark.parametrize("rows,cols", [(1, 256), (15, 512), (16, 1024), (17, 768), (255, 2048), (256, 1024), (257, 4096),
                                        (333, 3072), (1000, 14336), (4096, 1280), (70000, 1024)])
 def test_matvec_mma_kernel(fmt, batch, rows, cols):
-    # the batched tensor-core kernel (AUTO's choice for q8_0 / q4_0 / q4_K / q5_K / f16 from three columns on when cols is a
+    # the batched tensor-core kernel (AUTO's choice for every format but q6_K and q2_K from three columns on when cols is a
     # multiple of 256): ragged row counts around its 16-row fragments and 256-row stages, chunks of 256 / 512 / 1024 columns,
     # one and two groups of eight columns, more stages than CTAs (70000 rows) and fewer (1 row)
     lw.set_variant(lw.VARIANT_AUTO)
@@ -100,7 +100,7 @@ def test_matvec_mma_kernel(fmt, batch, rows, cols):
 
 
 @pytest.mark.parametrize("overlap", [0, 1, 2])
-@pytest.mark.parametrize("fmt", [lw.Q8_0, lw.Q4_0, lw.Q4_K, lw.Q5_K, lw.F16])
+@pytest.mark.parametrize("fmt", [lw.Q8_0, lw.Q4_0, lw.Q4_K, lw.Q5_K, lw.F16, lw.Q4_1, lw.Q5_0, lw.Q5_1])
 def test_matvec_mma_launch_modes(fmt, overlap):
     # the two ways the tensor-core kernel gets a cleared Y: one cooperative launch whose CTAs clear it and meet at a
     # grid barrier (no overlap), or a clearing kernel chained to it by programmatic dependent launch (overlap 1;
@@ -295,7 +295,7 @@ def test_matvec_group(variant, fmt, cols, row_list):
 
 @pytest.mark.parametrize("overlap", [0, 2])
 @pytest.mark.parametrize("batch", [2, 5, 12])
-@pytest.mark.parametrize("fmt", [lw.Q8_0, lw.Q4_0, lw.Q4_K, lw.Q5_K, lw.F16])
+@pytest.mark.parametrize("fmt", [lw.Q8_0, lw.Q4_0, lw.Q4_K, lw.Q5_K, lw.F16, lw.Q4_1, lw.Q5_0, lw.Q5_1])
 @pytest.mark.parametrize("cols,row_list,share", [(1024, [300, 77, 1000], True), (2048, [513, 256], True),
                                                  (768, [40, 1, 255, 17, 256, 3, 700, 64], False), (4096, [37], True)])
 def test_matvec_group_batch(fmt, batch, overlap, cols, row_list, share):
