@@ -54,14 +54,14 @@ MMA_FORMATS = ("q8_0", "q4_0", "q4_K", "q5_K", "f16", "q4_1", "q5_0", "q5_1")   
 def arithmetic_of(fmt, batch):
     """What the kernels compute in (the `dtype` key): not a precision claim, the arithmetic that runs."""
     if fmt == "f16" and batch >= 3:
-        return ("f32 in/out; f16 weights x three-term f16 split of the block-scaled fp32 activations on the tensor cores "
+        return ("f32 in/out; f16 weights x two-term f16 split of the block-scaled fp32 activations on the tensor cores "
                 "(mma m16n8k16), fp32 accumulation")
     if fmt == "f16":
         return "f32 in/out; f16 weights widened, fp32 FMA"
     if batch == 1:
         return "f32 in/out; activations as 24-bit block fixed point, int32 dp4a sums, fp32 block scales"
     if fmt in MMA_FORMATS and batch >= 3:
-        return ("f32 in/out; exact bf16 weight codes x three-term bf16 split of the fp32 activations on the tensor cores "
+        return ("f32 in/out; exact bf16 weight codes x two-term bf16 split (16 significant bits) of the fp32 activations on the tensor cores "
                 "(mma m16n8k16), fp32 accumulation and block scales")
     return "f32 in/out; batch > 1: per-column passes of the batch-1 kernel (24-bit block fixed point, int32 dp4a) or fp32 FMA tiles"
 
@@ -574,10 +574,10 @@ def run_step(args):
     }
     mma_served = batch > 1 and all(lw.query_variant(fmt_id, r, c, batch) == lw.VARIANT_MMA for _, r, c in shapes)
     if mma_served:
-        # the tensor-core kernel: every weight-column product is issued three times (one per bf16 term of the
+        # the tensor-core kernel: every weight-column product is issued twice (one per bf16 term of the
         # activation), in groups of eight columns; state the tensor work against the measured bf16 GEMM peak
         cols8 = 8 * ((batch + 7) // 8)
-        issued = sum(2.0 * r * c * cols8 * 3 for _, r, c in shapes)
+        issued = sum(2.0 * r * c * cols8 * 2 for _, r, c in shapes)
         try:
             with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as fh:
                 tpeak, tsrc = float(json.load(fh)["bf16_tflops_sustained"]), "measured (MEASURED_PEAKS.json bf16_tflops_sustained)"
@@ -586,7 +586,7 @@ def run_step(args):
         result["roofline_tensor"] = {
             "bound": "tensor", "achieved": round(issued / (step_ms * 1e-3) / 1e12, 1), "peak": tpeak, "peak_source": tsrc,
             "unit": "TFLOP/s", "frac": round(issued / (step_ms * 1e-3) / 1e12 / tpeak, 4),
-            "what": "bf16 products issued (3 terms x columns rounded up to 8) over the step time; the peak is the tcgen05 "
+            "what": "bf16 products issued (2 terms x columns rounded up to 8) over the step time; the peak is the tcgen05 "
                     "GEMM figure, which the warp-level mma used here cannot reach (measured: one m16n8k16 per ~10 cycles "
                     "per SM sub-partition, i.e. about 470 TFLOP/s for the whole GPU); the HBM roofline in `roofline` is the "
                     "bound a faster contraction would hit first"}

@@ -123,7 +123,7 @@ int lw_dequant(int fmt, const void* W_blocks, int64_t n, float* out, void* strea
  * huge compared with its neighbours and meets a weight that is zero or nearly so leaves an absolute error
  * that S does not cover.  For them
  *     E = c * sum_k What_k * A_k ,   c = 2^-18 (IDOT, the default for the quantised formats; MMA on q4_K / q5_K / q4_1 / q5_1), 2^-16 (STREAM),
- *                                    2^-30 (MMA on f16: activations as three f16 terms relative to their block's largest),
+ *                                    2^-30 (MMA on f16: activations as two f16 terms relative to their block's largest),
  * where, over the aligned run of 32 columns that contains k, A_k is the largest |x| and What_k the largest
  * decoded |w|.  This holds for weights made by lw_quantize, and for any block whose scale * code and offset
  * terms are at most four times its largest decoded magnitude.  The constants are worst-case figures (the
@@ -240,13 +240,15 @@ typedef enum {
                                is faster); forced, it runs passes of 8 and 4 columns */
     LW_VARIANT_MMA = 5      /* batch 2..16 only: tensor-core kernel (mma m16n8k16, bf16 operands, fp32 accumulation).
                                A weight's integer code is exact in bf16 and the block scale is applied in fp32 to each
-                               block's sum; every fp32 activation is cut into three bf16 terms that add up to it
-                               exactly, so E = 0 in the accuracy statement of lw_matvec for q8_0, q4_0 and q5_0.  q4_K,
-                               q5_K, q4_1 and q5_1 as well: there the codes are multiplied the same way, and the sub-block offsets
+                               block's sum; every fp32 activation is cut into two bf16 terms that add up to it within
+                               2^-16 of its magnitude (an error that scales with |w x| term by term and stays at
+                               0.15 of the tolerance at worst), so E = 0 in the accuracy statement of lw_matvec for
+                               q8_0, q4_0 and q5_0.  q4_K, q5_K, q4_1 and q5_1 as well: there the codes are
+                               multiplied the same way, and the sub-block offsets
                                (dmin * m) are applied to fp32 sums of each sub-block's activations, which brings the
                                extra term E back with c = 2^-18.  cols a multiple of 256; all columns in one pass
                                over the weights.  f16 as well: the weights are the A operand as they lie in
-                               memory, the activations three f16 terms of x * s with s a power of two per block of
+                               memory, the activations two f16 terms of x * s with s a power of two per block of
                                32 and column (E with c = 2^-30).  A row's sum is completed
                                with atomic additions (one per chunk of up to 1024 columns), so the last bits of a
                                result can differ from run to run.  AUTO takes it from 3 columns on */

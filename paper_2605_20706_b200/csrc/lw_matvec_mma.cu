@@ -8,10 +8,13 @@
 // to the narrow operand type:
 //   * the integer code of a weight (q - 8 in [-8, 7], resp. an int8) is exact in bf16; the fp16 block scale is
 //     applied in fp32 to each block's sum, as in the definition;
-//   * an fp32 activation is cut into three bf16 terms of eight significant bits each, by truncation:
-//     x = x1 + x2 + x3 exactly, so that code * x1 + code * x2 + code * x3, accumulated in fp32 by the tensor
-//     core, is the fp32-accumulated product with the exact activation.  A NaN or Inf stays one (in x1 or x2).
-// The accuracy is therefore that of the fp32 kernels: |y - y_ref| <= 1e-4 * sum|w x| + 1e-6 with no extra term
+//   * an fp32 activation is cut into two bf16 terms: x1 = x cut off after eight significant bits, x2 = the rest
+//     rounded to eight: x1 + x2 = x (1 + e) with |e| <= 2^-16, so code * x1 + code * x2, accumulated in fp32 by the
+//     tensor core, is the product with the activation to 2^-16 relative -- 0.15 of the tolerance if every term of a
+//     row erred the same way, and an error that scales with |w x| term by term (an activation that meets a zero
+//     weight contributes exactly nothing).  Three terms (x exactly, -DLW_MMA_TERMS=3) measured 13 % slower at 8
+//     columns and 23 % at 16, where the tensor pipe binds.  A NaN or Inf stays non-finite (in x1 or x2).
+// The accuracy is that of the fp32 kernels' contract: |y - y_ref| <= 1e-4 * sum|w x| + 1e-6 with no extra term
 // (q4_0, q8_0; q4_K's sub-block offsets go onto fp32 sums of the activations and bring an extra term back, see MmaQ4K).
 //
 // Why mma.sync and not tcgen05.mma here: the A operand is the decoded weight, which exists only in registers
@@ -27,7 +30,7 @@
 // units; a lane (g = lane / 4, t = lane % 4) reads word t of the quants of rows g and g + 8, which holds
 // exactly the eight weights of its A fragments once the k index inside a block is permuted -- the same
 // permutation is applied to the activations when a lane loads its B fragments, and a sum does not care.
-// The activations of a chunk of up to 1024 columns sit in shared memory as three bf16 planes.  Stages are
+// The activations of a chunk of up to 1024 columns sit in shared memory as one bf16 plane per term.  Stages are
 // numbered chunk-major, (row stage, sub-stage)-minor and dealt out in equal contiguous ranges to one CTA per
 // SM, so a matrix of few rows still keeps every SM busy; sums stay in registers while a CTA stays inside one
 // (chunk, row stage) and are then added into Y, which the host clears before the launch, with atomic adds
@@ -64,6 +67,10 @@ constexpr int kStageUnits = kStageCols / 64;
 constexpr int kMaxRing = 4;
 constexpr int kXPad = 64;                             // bytes after each column of a plane: 16-byte loads of lanes
                                                       // (g, t) at 64 g + 16 t cover 128 distinct bytes per quarter warp
+#ifndef LW_MMA_TERMS
+#define LW_MMA_TERMS 2
+#endif
+constexpr int kTerms = LW_MMA_TERMS;                  // terms an activation is cut into (planes in shared memory)
 constexpr int kSxBlockBytes = 64;                     // block sums of the activations: [block of 32][16 columns] floats
 constexpr int kMmaHeader = 128;                       // barriers, the stop flag and the grid barrier's generation
 constexpr uint32_t kGridPolls = 1u << 20;             // polls of the generation word (~0.5 us each) before giving up
@@ -418,10 +425,10 @@ struct MmaLegacy {
 // 256 columns are 512 bytes, fetched as four 128-byte slices (one per 64-column unit) with the 128-byte swizzle of
 // the tensor copy, so that the eight rows a warp reads at once fall into different banks: 16-byte chunk c of row r
 // of a slice sits at chunk c ^ (r % 8).  A stage is 128 rows; warps 0-7 take units 0 and 1 of their 16 rows, warps
-// 8-15 units 2 and 3.  The activations are held as three f16 terms of x * s, s a power of two per block of 32 and
-// column that brings the block's largest magnitude to 2^14..2^15: terms one and two are cut off exactly, the
-// third rounds what is left (at most 2^-38 of the block's largest magnitude is lost per element: the extra term E
-// of the accuracy statement with a tiny constant); 1 / s multiplies the block's sum.
+// 8-15 units 2 and 3.  The activations are held as f16 terms of x * s, s a power of two per block of 32 and
+// column that brings the block's largest magnitude to 2^14..2^15: the first term is cut off exactly, the second
+// rounds what is left (22 significant bits of the element, but nothing below 2^-38 of the block's largest
+// magnitude: the extra term E of the accuracy statement with a tiny constant); 1 / s multiplies the block's sum.
 struct MmaF16 {
     static constexpr int kStageRows = 128;
     static constexpr bool kF16 = true;
@@ -452,7 +459,7 @@ __device__ __forceinline__ void mma_f16_first(float (&d)[4], uint32_t a0, uint32
 // 0 (block 1: sw[2 + h]); sx = the lane's two block scales (1 / s), group nt 32 bytes further.
 template <int NT, int U, int BLK>
 __device__ __forceinline__ void block_step_f16(uint32_t wrow, const uint32_t (&sw)[4], uint32_t sx,
-                                               const uint32_t (&xp)[NT][3], float (&y)[NT][4]) {
+                                               const uint32_t (&xp)[NT][kTerms], float (&y)[NT][4]) {
     constexpr int kSlice = U * MmaF16::kSliceBytes;
     uint32_t a[4], b[4];
     lds64<kSlice>(wrow + sw[2 * BLK], a[0], a[1]);               // row g: k = 4t .. 4t+3
@@ -464,7 +471,7 @@ __device__ __forceinline__ void block_step_f16(uint32_t wrow, const uint32_t (&s
     for (int nt = 0; nt < NT; ++nt) {
         float c[4];
 #pragma unroll
-        for (int s = 0; s < 3; ++s) {
+        for (int s = 0; s < kTerms; ++s) {
             uint32_t b0, b1, b2, b3;
             lds128<kX>(xp[nt][s], b0, b1, b2, b3);
             if (s == 0)
@@ -493,7 +500,7 @@ __device__ __forceinline__ void block_step_f16(uint32_t wrow, const uint32_t (&s
 // activations, group nt 32 bytes further (formats with an offset term).
 template <class T, int NT, int U, int BLK>
 __device__ __forceinline__ void block_step(uint32_t wt, uint32_t row, uint32_t tabg, uint32_t sx,
-                                           const uint32_t (&xp)[NT][3], float (&y)[NT][4]) {
+                                           const uint32_t (&xp)[NT][kTerms], float (&y)[NT][4]) {
     constexpr int kPiece = T::kPiece;
     uint32_t a[4], b[4];
     const int t = (int)((wt - row) >> 2);
@@ -507,7 +514,7 @@ __device__ __forceinline__ void block_step(uint32_t wt, uint32_t row, uint32_t t
     for (int nt = 0; nt < NT; ++nt) {
         float c[4];
 #pragma unroll
-        for (int s = 0; s < 3; ++s) {
+        for (int s = 0; s < kTerms; ++s) {
             uint32_t b0, b1, b2, b3;
             lds128<kX>(xp[nt][s], b0, b1, b2, b3);      // k = 4t .. 4t+3 and k = 16+4t .. 16+4t+3
             if (s == 0)
@@ -535,24 +542,35 @@ __device__ __forceinline__ void block_step(uint32_t wt, uint32_t row, uint32_t t
     }
 }
 
-// fp32 -> three bf16 terms by truncation (x1 + x2 + x3 == x exactly; the differences are exact in fp32)
+// fp32 -> bf16 terms.  The first is x cut off after eight significant bits (exact difference).  With two terms
+// (the default) the second is the rest rounded to nearest: x1 + x2 = x (1 + e), |e| <= 2^-16.  With three
+// (-DLW_MMA_TERMS=3) the second is cut off as well and the third holds what is left: x1 + x2 + x3 == x exactly.
+// A NaN stays one (in x1, or in x2 when only its low payload bits were set); an Inf gives x2 = NaN.
 __device__ __forceinline__ void split3(float x, uint32_t& h1, uint32_t& h2, uint32_t& h3) {
     const uint32_t b1 = __float_as_uint(x) & 0xFFFF0000u;
     const float r1 = x - __uint_as_float(b1);
-    const uint32_t b2 = __float_as_uint(r1) & 0xFFFF0000u;
-    const float r2 = r1 - __uint_as_float(b2);
     h1 = b1 >> 16;
-    h2 = b2 >> 16;
-    h3 = __float_as_uint(r2) >> 16;                     // at most eight significant bits are left: exact
+    if (kTerms == 2) {
+        unsigned short r;
+        asm("cvt.rn.bf16.f32 %0, %1;" : "=h"(r) : "f"(r1));
+        h2 = r;
+        h3 = 0;
+    } else {
+        const uint32_t b2 = __float_as_uint(r1) & 0xFFFF0000u;
+        const float r2 = r1 - __uint_as_float(b2);
+        h2 = b2 >> 16;
+        h3 = __float_as_uint(r2) >> 16;                 // at most eight significant bits are left: exact
+    }
 }
 
-// fp32 -> three f16 terms of x (already scaled into the f16 range): the first two cut off (exact differences), the
-// third rounds the rest
+// fp32 -> f16 terms of x (already scaled into the f16 range): cut off (exact differences) except the last, which
+// rounds the rest
 __device__ __forceinline__ void split3_f16(float x, uint32_t& h1, uint32_t& h2, uint32_t& h3) {
     unsigned short a, b, c;
     asm("cvt.rz.f16.f32 %0, %1;" : "=h"(a) : "f"(x));
     const float r1 = x - __half2float(__ushort_as_half(a));
-    asm("cvt.rz.f16.f32 %0, %1;" : "=h"(b) : "f"(r1));
+    if (kTerms == 2) asm("cvt.rn.f16.f32 %0, %1;" : "=h"(b) : "f"(r1));
+    else asm("cvt.rz.f16.f32 %0, %1;" : "=h"(b) : "f"(r1));
     const float r2 = r1 - __half2float(__ushort_as_half(b));
     asm("cvt.rn.f16.f32 %0, %1;" : "=h"(c) : "f"(r2));
     h1 = a, h2 = b, h3 = c;
@@ -777,7 +795,7 @@ __global__ void __launch_bounds__(kMmaThreads, kCtasPerSm) matvec_mma_kernel(con
             cur_it = cur.it;
         }
         if (c != cur_c || mat.X != cur_x) {
-            // the chunk's activations as three bf16 planes: plane s, column b.  Inside a block of 32 the order is
+            // the chunk's activations as one bf16 (f16) plane per term: plane s, column b.  Inside a block of 32 the order is
             // the one the fragments want: slots 8 q .. 8 q + 3 hold k = 4 q .. 4 q + 3 and slots 8 q + 4 .. 8 q + 7
             // hold k = 16 + 4 q .., so a lane reads both halves of its B operand with one 16-byte load.
             cur_c = c;
@@ -847,7 +865,7 @@ __global__ void __launch_bounds__(kMmaThreads, kCtasPerSm) matvec_mma_kernel(con
                         const int slot4 = (k4 & ~7) + 2 * (k4 & 3) + ((k4 >> 2) & 1);    // quad of slots the quad of k goes to
                         const uint32_t dst = xs + b * x_pitch + 8u * slot4;
 #pragma unroll
-                        for (int s = 0; s < 3; ++s)
+                        for (int s = 0; s < kTerms; ++s)
                             asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(dst + s * plane_pitch),
                                          "r"(h[s][0] | (h[s][1] << 16)), "r"(h[s][2] | (h[s][3] << 16))
                                          : "memory");
@@ -871,11 +889,11 @@ __global__ void __launch_bounds__(kMmaThreads, kCtasPerSm) matvec_mma_kernel(con
                 T::prepare(row - (uint32_t)g * kPiece, tab, lane);
                 __syncwarp();
             }
-            uint32_t xp[NT][3];
+            uint32_t xp[NT][kTerms];
 #pragma unroll
             for (int nt = 0; nt < NT; ++nt)
 #pragma unroll
-                for (int s = 0; s < 3; ++s)
+                for (int s = 0; s < kTerms; ++s)
                     xp[nt][s] = xlane + 2u * (uint32_t)(j * kStageCols) + s * plane_pitch + nt * 8 * x_pitch;
             if constexpr (T::kF16) {
                 const uint32_t wr = wrow + (uint32_t)slot * kStageBytes;
@@ -1001,7 +1019,7 @@ bool mma_plan(int fmt, int64_t cols, int nt, int& chunk_cols, int& ring, size_t&
     // 1024 columns and two 68 KB stages against 0.49 ms with chunks of 256 and three)
     for (int kx = 1024; kx >= 256; kx /= 2) {
         if (cols % kx != 0) continue;
-        x_bytes = (size_t)3 * 8 * nt * (2 * kx + kXPad);
+        x_bytes = (size_t)kTerms * 8 * nt * (2 * kx + kXPad);
         if (x_bytes + 2 * stage_bytes > budget) continue;
         size_t n = (budget - x_bytes) / stage_bytes;
         ring = (int)(n > (size_t)kMaxRing ? kMaxRing : n);

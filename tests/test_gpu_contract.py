@@ -98,7 +98,7 @@ def test_outliers_on_zero_weights_stay_inside_the_stated_bound(fmt, variant, zer
                                         (lw.Q4_0, lw.VARIANT_MMA), (lw.Q5_0, lw.VARIANT_MMA)])
 def test_batched_kernels_need_no_extra_term(fmt, kernel):
     # the batched fp32 tile kernel decodes every weight exactly before it multiplies, and the tensor-core kernel
-    # multiplies exact integer codes with three bf16 terms that add up to the activation exactly: the plain
+    # multiplies exact integer codes with two bf16 terms that add up to the activation within 2^-16: the plain
     # tolerance holds on the same adversarial activations (eight columns, each with its own outliers), as the
     # header states
     rows, cols, batch = 48, 4096, 8
@@ -119,7 +119,7 @@ def test_batched_kernels_need_no_extra_term(fmt, kernel):
         Xb[3, 100] = bad
         y = _run(fmt, blocks, rows, cols, Xb, kernel, batch)
         assert not np.isfinite(y[3]).any() and np.isfinite(np.delete(y, 3, axis=0)).all()
-    # extreme magnitudes survive the three-term split: a huge value (the sums of code * x stay finite up to about
+    # extreme magnitudes survive the split into terms: a huge value (the sums of code * x stay finite up to about
     # 2^115, the limit the header states for the batched kernels) and a denormal
     Xe = np.zeros((batch, cols), np.float32)
     Xe[0, 7] = 1e30
@@ -136,7 +136,7 @@ def test_batched_kernels_need_no_extra_term(fmt, kernel):
 def test_formats_with_an_extra_term_on_the_tensor_cores_stay_inside_the_stated_bound(fmt, c_extra):
     # q4_K / q5_K in the batched tensor-core kernel apply the sub-block offsets to sums of activations, like the
     # fp32-activation streaming family: the header gives them the extra term with c = 2^-18; f16 holds the
-    # activations as three f16 terms relative to each block's largest magnitude, which can lose up to 2^-38 of that
+    # activations as two f16 terms relative to each block's largest magnitude, which can lose up to 2^-38 of that
     # magnitude per element (c = 2^-30 stated).  Asserted here on the adversarial activations (eight columns, each
     # with its own outliers); a non-finite activation stays in its column
     rows, cols, batch = 48, 4096, 8
