@@ -103,7 +103,7 @@ int lw_dequant(int fmt, const void* W_blocks, int64_t n, float* out, void* strea
 
 /* Fused dequantise + mat-vec [Sec 3.2, 3.3]: Y[b*rows + r] = sum_k decode(W)[r][k] * X[b*cols + k],
  * fp32 accumulation, for b < batch (1..16).  The batched kernels reuse every decoded block for all
- * their columns: without a forced variant every format but q6_K and q2_K, with cols a multiple of 256, runs on the tensor
+ * their columns: without a forced variant every format but q2_K, with cols a multiple of 256 (q6_K: of 2048), runs on the tensor
  * cores from three columns on (LW_VARIANT_MMA); the other quantised formats (and f16 up to four columns)
  * run one streaming pass per column instead (four columns per launch), which measures faster on B200
  * than their batched kernels.
@@ -115,7 +115,7 @@ int lw_dequant(int fmt, const void* W_blocks, int64_t n, float* out, void* strea
  * Accuracy.  With w the decoded weights and S = sum_k |w_k x_k|, every result satisfies
  *     |y - y_exact| <= 1e-4 * S + 1e-6 + E .
  * E = 0 for LW_VARIANT_GENERIC and for f16 at batch 1 and 2 (each weight is decoded exactly and then multiplied:
- * plain fp32 accumulation), for any finite input, and for the batched LW_VARIANT_TILE and LW_VARIANT_MMA on q8_0, q4_0, q5_0
+ * plain fp32 accumulation), for any finite input, and for the batched LW_VARIANT_TILE and LW_VARIANT_MMA on q8_0, q4_0, q5_0, q6_K
  * (exact integer codes times exact activations, block sums scaled in fp32) as long as |x| <= 2^115, which keeps a
  * block's sum of code * x finite.  The streaming variants multiply the integer codes first and apply
  * block scales and offsets to the sums, and LW_VARIANT_IDOT holds the activations as block fixed point
@@ -158,7 +158,7 @@ typedef struct {
 int lw_matvec_group(int fmt, int64_t cols, int n_items, const lw_group_item* items, void* stream);
 
 /* The same with `batch` activation columns per item (1..16): X of an item is batch * cols floats, Y batch * rows
- * floats, laid out as in lw_matvec.  batch 1 is lw_matvec_group.  From two columns on, every format but q6_K and q2_K with cols a
+ * floats, laid out as in lw_matvec.  batch 1 is lw_matvec_group.  From two columns on, every format but q2_K with cols a
  * multiple of 256 run all items in ONE launch of the tensor-core kernel (LW_VARIANT_MMA, unless another variant
  * is forced; items that follow one another and share their X pointer share its converted copy); everything else
  * is run item by item with lw_matvec.  Errors as lw_matvec (LW_ERR_BATCH for batch outside 1..16); a call that
@@ -243,7 +243,7 @@ typedef enum {
                                block's sum; every fp32 activation is cut into two bf16 terms that add up to it within
                                2^-16 of its magnitude (an error that scales with |w x| term by term and stays at
                                0.15 of the tolerance at worst), so E = 0 in the accuracy statement of lw_matvec for
-                               q8_0, q4_0 and q5_0.  q4_K, q5_K, q4_1 and q5_1 as well: there the codes are
+                               q8_0, q4_0, q5_0 and q6_K (cols a multiple of 2048).  q4_K, q5_K, q4_1 and q5_1 as well: there the codes are
                                multiplied the same way, and the sub-block offsets
                                (dmin * m) are applied to fp32 sums of each sub-block's activations, which brings the
                                extra term E back with c = 2^-18.  cols a multiple of 256; all columns in one pass

@@ -1,4 +1,4 @@
-// Batched mat-vec on the tensor cores (batch 2..16; q4_0, q8_0, q4_K, q5_K, q4_1, q5_0, q5_1 and f16) [paper Sec 3.2: from a handful of columns on
+// Batched mat-vec on the tensor cores (batch 2..16; every format but q2_K) [paper Sec 3.2: from a handful of columns on
 // the mat-vec turns into a small mat-mat product, a dense contraction; Sec 3.3: one decode routine per format
 // spliced into a common skeleton].
 //
@@ -192,6 +192,7 @@ __device__ __forceinline__ uint32_t bytes_to_bf16_128_plus(uint32_t v) {
 struct MmaQ40 {
     static constexpr int kStageRows = 256;          // 16 warps x 16 rows
     static constexpr bool kF16 = false;
+    static constexpr bool kQ6K = false;
     static constexpr int kPiece = 8 * 18;               // bytes of a row's 256 columns
     static constexpr bool kHasMin = false;              // no per-block offset term
     static constexpr int kTableBytes = 0;               // no per-warp table of decoded scales
@@ -222,6 +223,7 @@ struct MmaQ40 {
 struct MmaQ80 {
     static constexpr int kStageRows = 256;          // 16 warps x 16 rows
     static constexpr bool kF16 = false;
+    static constexpr bool kQ6K = false;
     static constexpr int kPiece = 8 * 34;
     static constexpr bool kHasMin = false;
     static constexpr int kTableBytes = 0;
@@ -263,6 +265,7 @@ struct MmaQ80 {
 struct MmaQ4K {
     static constexpr int kStageRows = 256;          // 16 warps x 16 rows
     static constexpr bool kF16 = false;
+    static constexpr bool kQ6K = false;
     static constexpr int kPiece = 144;
     static constexpr bool kHasMin = true;
     static constexpr int kTableBytes = 16 * 8 * 8;      // per warp: 16 rows x 8 sub-blocks x (d * sc, dmin * m)
@@ -317,6 +320,7 @@ struct MmaQ4K {
 struct MmaQ5K {
     static constexpr int kStageRows = 256;          // 16 warps x 16 rows
     static constexpr bool kF16 = false;
+    static constexpr bool kQ6K = false;
     static constexpr int kPiece = 176;
     static constexpr bool kHasMin = true;
     static constexpr int kTableBytes = MmaQ4K::kTableBytes;
@@ -379,6 +383,7 @@ struct MmaLegacy {
     static constexpr int kBlock = FMT == LW_Q4_1 ? 20 : (FMT == LW_Q5_0 ? 22 : 24);
     static constexpr int kStageRows = 256;
     static constexpr bool kF16 = false;
+    static constexpr bool kQ6K = false;
     static constexpr int kPiece = 8 * kBlock;
     static constexpr int kTableBytes = 0;
     static __device__ __forceinline__ void prepare(uint32_t, uint32_t, int) {}
@@ -432,6 +437,7 @@ struct MmaLegacy {
 struct MmaF16 {
     static constexpr int kStageRows = 128;
     static constexpr bool kF16 = true;
+    static constexpr bool kQ6K = false;
     static constexpr int kPiece = 512;
     static constexpr bool kHasMin = false;
     static constexpr int kTableBytes = 0;
@@ -490,6 +496,111 @@ __device__ __forceinline__ void block_step_f16(uint32_t wrow, const uint32_t (&s
         y[nt][2] = fmaf(s0, c[2], y[nt][2]);
         y[nt][3] = fmaf(s1, c[3], y[nt][3]);
     }
+}
+
+// q6_K: 210-byte super-blocks {128 bytes of low nibbles, 64 bytes of upper bit pairs, 16 int8 scales (one per 16
+// weights), d}.  210 is not a multiple of 16, so a row's piece of a stage starts anywhere on a 2-byte grid: the
+// tensor copy starts at the 16-byte boundary below it and fetches 224 bytes per row, and the kernel indexes from
+// the remainder `o` (0, 2, .. 14); where o is 2 modulo 4 every word of the piece straddles two words of shared
+// memory (MIS: two loads and a byte permute).  A code is nibble | two upper bits << 4 = 0..63, minus 32: exact in
+// bf16, and there is no offset term: E = 0.  The two 16-weight halves of a block have their own scales, so the two
+// mma of a term go to separate accumulators.  Unit U = half U / 2 of the super-block, groups {0, 1} (low nibbles of
+// bytes l and l + 32) for even U and {2, 3} (high nibbles) for odd U.
+struct MmaQ6K {
+    static constexpr int kStageRows = 256;
+    static constexpr bool kF16 = false;
+    static constexpr bool kQ6K = true;
+    static constexpr int kPiece = 224;                  // bytes fetched per row and stage (210 + up to 14 in front)
+    static constexpr bool kHasMin = false;
+    static constexpr int kTableBytes = 16 * 16 * 4;     // per warp: 16 rows x 16 (d * scale)
+    // rows = the warp's first row piece + o; lane: row lane / 2, scales 8 (lane % 2) .. + 7
+    static __device__ __forceinline__ void prepare(uint32_t rows, uint32_t tab, int lane) {
+        const uint32_t row = rows + (uint32_t)(lane >> 1) * kPiece;
+        const float d = lds_half<208>(row);
+        const uint32_t sc = row + 192u + 8u * (lane & 1), out = tab + (uint32_t)(lane >> 1) * 64u + 32u * (lane & 1);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            int v;
+            asm volatile("ld.shared.s8 %0, [%1];" : "=r"(v) : "r"(sc + j));
+            asm volatile("st.shared.f32 [%0], %1;" ::"r"(out + 4u * j), "f"(d * (float)v) : "memory");
+        }
+    }
+};
+
+// A 32-bit word of the piece at byte OFF from `wt` (word-aligned address below the piece's word + 4 t); MIS: the piece
+// is two bytes off the word grid.
+template <int OFF, bool MIS>
+__device__ __forceinline__ uint32_t q6k_word(uint32_t wt) {
+    if (MIS) return __byte_perm(lds32<OFF>(wt), lds32<OFF + 4>(wt), 0x5432u);
+    return lds32<OFF>(wt);
+}
+
+// One group of 32 q6_K weights of the warp's 16 rows against all columns.  tabg = the warp's table at row g.
+template <int NT, int U, int BLK, bool MIS>
+__device__ __forceinline__ void block_step_q6k(uint32_t wt, uint32_t tabg, const uint32_t (&xp)[NT][kTerms],
+                                               float (&y)[NT][4]) {
+    constexpr int kHalf = U / 2, kGroup = 2 * (U & 1) + BLK;
+    constexpr int kQl = 64 * kHalf + 32 * BLK, kQh = 128 + 32 * kHalf, kShift = 2 * kGroup;
+    constexpr bool kHigh = (U & 1) != 0;
+    constexpr int kRow8 = 8 * MmaQ6K::kPiece;
+    uint32_t a[4], b[4];
+    {
+        const uint32_t bias = 0x43204320u;              // (160, 160): (128 + code) - 160 = code - 32, exactly
+        uint32_t l0 = q6k_word<kQl, MIS>(wt), l1 = q6k_word<kQl + 16, MIS>(wt);
+        uint32_t h0 = q6k_word<kQh, MIS>(wt), h1 = q6k_word<kQh + 16, MIS>(wt);
+        if (kHigh) l0 >>= 4, l1 >>= 4;
+        l0 = (l0 & 0x0F0F0F0Fu) | (((h0 >> kShift) & 0x03030303u) << 4);
+        l1 = (l1 & 0x0F0F0F0Fu) | (((h1 >> kShift) & 0x03030303u) << 4);
+        a[0] = sub_bf16x2(bytes_to_bf16_128_plus<0>(l0), bias);
+        a[1] = sub_bf16x2(bytes_to_bf16_128_plus<2>(l0), bias);
+        a[2] = sub_bf16x2(bytes_to_bf16_128_plus<0>(l1), bias);
+        a[3] = sub_bf16x2(bytes_to_bf16_128_plus<2>(l1), bias);
+        l0 = q6k_word<kRow8 + kQl, MIS>(wt), l1 = q6k_word<kRow8 + kQl + 16, MIS>(wt);
+        h0 = q6k_word<kRow8 + kQh, MIS>(wt), h1 = q6k_word<kRow8 + kQh + 16, MIS>(wt);
+        if (kHigh) l0 >>= 4, l1 >>= 4;
+        l0 = (l0 & 0x0F0F0F0Fu) | (((h0 >> kShift) & 0x03030303u) << 4);
+        l1 = (l1 & 0x0F0F0F0Fu) | (((h1 >> kShift) & 0x03030303u) << 4);
+        b[0] = sub_bf16x2(bytes_to_bf16_128_plus<0>(l0), bias);
+        b[1] = sub_bf16x2(bytes_to_bf16_128_plus<2>(l0), bias);
+        b[2] = sub_bf16x2(bytes_to_bf16_128_plus<0>(l1), bias);
+        b[3] = sub_bf16x2(bytes_to_bf16_128_plus<2>(l1), bias);
+    }
+    float s00, s01, s10, s11;                            // d * scale of (row g, half 0 / 1), (row g + 8, half 0 / 1)
+    lds_f32x2<4 * (8 * kHalf + 2 * kGroup)>(tabg, s00, s01);
+    lds_f32x2<8 * 64 + 4 * (8 * kHalf + 2 * kGroup)>(tabg, s10, s11);
+    constexpr int kX = 2 * (64 * U + 32 * BLK);
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+        float c0[4], c1[4];
+#pragma unroll
+        for (int s = 0; s < kTerms; ++s) {
+            uint32_t b0, b1, b2, b3;
+            lds128<kX>(xp[nt][s], b0, b1, b2, b3);
+            if (s == 0) {
+                mma_bf16_first(c0, a[0], b[0], a[1], b[1], b0, b1);
+                mma_bf16_first(c1, a[2], b[2], a[3], b[3], b2, b3);
+            } else {
+                mma_bf16(c0, a[0], b[0], a[1], b[1], b0, b1);
+                mma_bf16(c1, a[2], b[2], a[3], b[3], b2, b3);
+            }
+        }
+        y[nt][0] = fmaf(s01, c1[0], fmaf(s00, c0[0], y[nt][0]));
+        y[nt][1] = fmaf(s01, c1[1], fmaf(s00, c0[1], y[nt][1]));
+        y[nt][2] = fmaf(s11, c1[2], fmaf(s10, c0[2], y[nt][2]));
+        y[nt][3] = fmaf(s11, c1[3], fmaf(s10, c0[3], y[nt][3]));
+    }
+}
+
+template <int NT, bool MIS>
+__device__ __forceinline__ void stage_q6k(uint32_t wt, uint32_t tabg, const uint32_t (&xp)[NT][kTerms], float (&y)[NT][4]) {
+    block_step_q6k<NT, 0, 0, MIS>(wt, tabg, xp, y);
+    block_step_q6k<NT, 0, 1, MIS>(wt, tabg, xp, y);
+    block_step_q6k<NT, 1, 0, MIS>(wt, tabg, xp, y);
+    block_step_q6k<NT, 1, 1, MIS>(wt, tabg, xp, y);
+    block_step_q6k<NT, 2, 0, MIS>(wt, tabg, xp, y);
+    block_step_q6k<NT, 2, 1, MIS>(wt, tabg, xp, y);
+    block_step_q6k<NT, 3, 0, MIS>(wt, tabg, xp, y);
+    block_step_q6k<NT, 3, 1, MIS>(wt, tabg, xp, y);
 }
 
 // One block (32 weights) of the warp's 16 rows against all columns: decode the lane's fragments of rows g and
@@ -689,6 +800,11 @@ __global__ void __launch_bounds__(kMmaThreads, kCtasPerSm) matvec_mma_kernel(con
                     tensor_load_2d(smem + p.w_off + (size_t)cur.slot * kStageBytes + u * MmaF16::kSliceBytes,
                                    &maps.m[cur.it], ((cur.c * spc + cur.j) * 4 + u) * 32,
                                    (cur.rs - p.item[cur.it].rs_begin) * kStageRows, &full[cur.slot], policy);
+            } else if constexpr (T::kQ6K) {
+                // the piece starts at byte 210 * (stage's column index) of the row: fetch from the 16-byte boundary below
+                tensor_load_2d(smem + p.w_off + (size_t)cur.slot * kStageBytes, &maps.m[cur.it],
+                               ((210 * (cur.c * spc + cur.j)) >> 4) << 2, (cur.rs - p.item[cur.it].rs_begin) * kStageRows,
+                               &full[cur.slot], policy);
             } else {
                 tensor_load_2d(smem + p.w_off + (size_t)cur.slot * kStageBytes, &maps.m[cur.it],
                                (cur.c * spc + cur.j) * (kPiece / 4), (cur.rs - p.item[cur.it].rs_begin) * kStageRows,
@@ -885,7 +1001,11 @@ __global__ void __launch_bounds__(kMmaThreads, kCtasPerSm) matvec_mma_kernel(con
             const uint32_t row = wrow + (uint32_t)slot * kStageBytes, wt = row + 4u * t;
             const uint32_t tab = smem_u32(smem + p.tab_off) + (uint32_t)warp * T::kTableBytes, tabg = tab + 64u * g;
             const uint32_t sx = smem_u32(smem + p.sx_off) + (uint32_t)(8 * j) * kSxBlockBytes + 8u * t;
-            if constexpr (T::kTableBytes > 0) {
+            if constexpr (T::kQ6K) {
+                const uint32_t o = (uint32_t)(210 * (c * spc + j)) & 15u;      // the piece's offset in the fetched bytes
+                T::prepare(row - (uint32_t)g * kPiece + o, tab, lane);
+                __syncwarp();
+            } else if constexpr (T::kTableBytes > 0) {
                 T::prepare(row - (uint32_t)g * kPiece, tab, lane);
                 __syncwarp();
             }
@@ -895,7 +1015,13 @@ __global__ void __launch_bounds__(kMmaThreads, kCtasPerSm) matvec_mma_kernel(con
 #pragma unroll
                 for (int s = 0; s < kTerms; ++s)
                     xp[nt][s] = xlane + 2u * (uint32_t)(j * kStageCols) + s * plane_pitch + nt * 8 * x_pitch;
-            if constexpr (T::kF16) {
+            if constexpr (T::kQ6K) {
+                const uint32_t o = (uint32_t)(210 * (c * spc + j)) & 15u;
+                if (o & 2u)
+                    stage_q6k<NT, true>(wt + (o & ~3u), tabg, xp, y);
+                else
+                    stage_q6k<NT, false>(wt + o, tabg, xp, y);
+            } else if constexpr (T::kF16) {
                 const uint32_t wr = wrow + (uint32_t)slot * kStageBytes;
                 if (warp < 8) {
                     block_step_f16<NT, 0, 0>(wr, sw, sx, xp, y);
@@ -1007,10 +1133,11 @@ bool mma_plan(int fmt, int64_t cols, int nt, int& chunk_cols, int& ring, size_t&
                       : fmt == LW_Q4_1 ? MmaLegacy<LW_Q4_1>::kPiece
                       : fmt == LW_Q5_0 ? MmaLegacy<LW_Q5_0>::kPiece
                       : fmt == LW_Q5_1 ? MmaLegacy<LW_Q5_1>::kPiece
+                      : fmt == LW_Q6_K ? MmaQ6K::kPiece
                                        : MmaF16::kPiece;
     stage_bytes = (size_t)mma_stage_rows(fmt) * piece;
     // q4_K: block sums of the activations (64 bytes per block of a chunk of up to 1024 columns) and the warps' tables
-    extra_bytes = (fmt == LW_Q4_K || fmt == LW_Q5_K)
+    extra_bytes = (fmt == LW_Q4_K || fmt == LW_Q5_K || fmt == LW_Q6_K)
                       ? (size_t)(1024 / 32) * kSxBlockBytes + (size_t)kMmaWarps * MmaQ4K::kTableBytes
                       : ((fmt == LW_F16 || fmt == LW_Q4_1 || fmt == LW_Q5_1) ? (size_t)(1024 / 32) * kSxBlockBytes : 0);
     // (f16: up to 1 KB more goes into aligning the swizzled stages)
@@ -1033,8 +1160,9 @@ bool mma_plan(int fmt, int64_t cols, int nt, int& chunk_cols, int& ring, size_t&
 
 bool matvec_mma_supported(int fmt, int64_t rows, int64_t cols, int batch) {
     if (fmt != LW_Q4_0 && fmt != LW_Q8_0 && fmt != LW_Q4_K && fmt != LW_Q5_K && fmt != LW_F16 && fmt != LW_Q4_1 &&
-        fmt != LW_Q5_0 && fmt != LW_Q5_1)
+        fmt != LW_Q5_0 && fmt != LW_Q5_1 && fmt != LW_Q6_K)
         return false;
+    if (fmt == LW_Q6_K && cols % 2048 != 0) return false;      // 210-byte super-blocks: rows must be whole 16-byte units
     if (batch < 2 || batch > 16) return false;
     if (cols % kStageCols != 0) return false;
     return rows >= 1 && rows <= (int64_t)1 << 30;
@@ -1123,7 +1251,7 @@ int launch_matvec_mma_group(int fmt, int64_t cols, int n_items, const void* cons
     p.grid_bar = grid_bar;
     p.x_off = kMmaHeader;
     p.sx_off = (uint32_t)(kMmaHeader + x_bytes);
-    p.tab_off = p.sx_off + (uint32_t)((fmt == LW_Q4_K || fmt == LW_Q5_K) ? (1024 / 32) * kSxBlockBytes : 0);
+    p.tab_off = p.sx_off + (uint32_t)((fmt == LW_Q4_K || fmt == LW_Q5_K || fmt == LW_Q6_K) ? (1024 / 32) * kSxBlockBytes : 0);
     // the stages: 128-byte aligned; f16's swizzle pattern is one of address bits, so its stages start on 1 KB
     const size_t w_align = fmt == LW_F16 ? 1024 : 128;
     p.w_off = (uint32_t)((kMmaHeader + x_bytes + extra_bytes + w_align - 1) / w_align * w_align);
@@ -1152,6 +1280,9 @@ int launch_matvec_mma_group(int fmt, int64_t cols, int n_items, const void* cons
     if (fmt == LW_F16)
         return nt == 1 ? launch_mma<MmaF16, 1>(p, maps, grid, smem_bytes, overlap != 0, stream)
                        : launch_mma<MmaF16, 2>(p, maps, grid, smem_bytes, overlap != 0, stream);
+    if (fmt == LW_Q6_K)
+        return nt == 1 ? launch_mma<MmaQ6K, 1>(p, maps, grid, smem_bytes, overlap != 0, stream)
+                       : launch_mma<MmaQ6K, 2>(p, maps, grid, smem_bytes, overlap != 0, stream);
     if (fmt == LW_Q4_1)
         return nt == 1 ? launch_mma<MmaLegacy<LW_Q4_1>, 1>(p, maps, grid, smem_bytes, overlap != 0, stream)
                        : launch_mma<MmaLegacy<LW_Q4_1>, 2>(p, maps, grid, smem_bytes, overlap != 0, stream);

@@ -95,7 +95,7 @@ def test_outliers_on_zero_weights_stay_inside_the_stated_bound(fmt, variant, zer
 
 
 @pytest.mark.parametrize("fmt,kernel", [(lw.Q8_0, lw.VARIANT_TILE), (lw.Q4_0, lw.VARIANT_TILE), (lw.Q8_0, lw.VARIANT_MMA),
-                                        (lw.Q4_0, lw.VARIANT_MMA), (lw.Q5_0, lw.VARIANT_MMA)])
+                                        (lw.Q4_0, lw.VARIANT_MMA), (lw.Q5_0, lw.VARIANT_MMA), (lw.Q6_K, lw.VARIANT_MMA)])
 def test_batched_kernels_need_no_extra_term(fmt, kernel):
     # the batched fp32 tile kernel decodes every weight exactly before it multiplies, and the tensor-core kernel
     # multiplies exact integer codes with two bf16 terms that add up to the activation within 2^-16: the plain

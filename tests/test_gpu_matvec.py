@@ -84,7 +84,7 @@ def test_matvec_tile_kernel(fmt, batch, rows, cols):
 @pytest.mark.parametrize("rows,cols", [(1, 256), (15, 512), (16, 1024), (17, 768), (255, 2048), (256, 1024), (257, 4096),
                                        (333, 3072), (1000, 14336), (4096, 1280), (70000, 1024)])
 def test_matvec_mma_kernel(fmt, batch, rows, cols):
-    # the batched tensor-core kernel (AUTO's choice for every format but q6_K and q2_K from three columns on when cols is a
+    # the batched tensor-core kernel (AUTO's choice for every format but q2_K (q6_K: its own test) from three columns on when cols is a
     # multiple of 256): ragged row counts around its 16-row fragments and 256-row stages, chunks of 256 / 512 / 1024 columns,
     # one and two groups of eight columns, more stages than CTAs (70000 rows) and fewer (1 row)
     lw.set_variant(lw.VARIANT_AUTO)
@@ -97,6 +97,33 @@ def test_matvec_mma_kernel(fmt, batch, rows, cols):
     check_matvec(y, y_ref, s_ref, "mma fmt %d %dx%d batch %d" % (fmt, rows, cols, batch))
     y = gpu_matvec(fmt, blocks, rows, cols, X, batch, lw.VARIANT_AUTO)
     check_matvec(y, y_ref, s_ref, "auto fmt %d %dx%d batch %d" % (fmt, rows, cols, batch))
+
+
+@pytest.mark.parametrize("batch", [3, 8, 13, 16])
+@pytest.mark.parametrize("rows,cols", [(1, 2048), (17, 2048), (255, 4096), (300, 6144), (513, 14336), (4096, 2048)])
+def test_matvec_mma_kernel_q6_K(batch, rows, cols):
+    # q6_K on the tensor cores: 210-byte super-blocks, so a stage's row pieces start on a 2-byte grid inside the
+    # 16-byte-aligned fetch (all eight remainders occur from 16 column stages on, the odd ones with straddled
+    # words); cols must be a multiple of 2048
+    fmt = lw.Q6_K
+    lw.set_variant(lw.VARIANT_AUTO)
+    assert lw.query_variant(fmt, rows, cols, batch) == lw.VARIANT_MMA
+    assert lw.query_variant(fmt, rows, cols + 256, batch) != lw.VARIANT_MMA
+    blocks = quantized_weights(fmt, rows, cols, seed=66, tensor_id=fmt, outlier_p=0.01)
+    X = synth.activations(66, batch, batch, cols)
+    y_ref, s_ref = oracle.matvec(fmt, blocks, rows, cols, X, batch, nthreads=8)
+    y = gpu_matvec(fmt, blocks, rows, cols, X, batch, lw.VARIANT_AUTO)
+    check_matvec(y, y_ref, s_ref, "mma q6_K %dx%d batch %d" % (rows, cols, batch))
+    # and two matrices in one launch
+    w = torch.from_numpy(blocks).cuda()
+    x = torch.from_numpy(X).cuda()
+    ys = [Guarded((batch, rows)), Guarded((batch, rows))]
+    lw.matvec_group(fmt, cols, [(w, rows, x, ys[0].t), (w, rows, x, ys[1].t)], batch=batch)
+    torch.cuda.synchronize()
+    for yg in ys:
+        yg.check("grouped Y")
+        check_matvec(yg.t.cpu().numpy(), y_ref, s_ref, "grouped mma q6_K")
+    assert lw.device_status() == 0
 
 
 @pytest.mark.parametrize("overlap", [0, 1, 2])

@@ -144,7 +144,8 @@ def test_variant_controls():
     assert lw.query_variant(lw.Q4_K, 4096, 4096, 8) == lw.VARIANT_MMA         # q4_K as well (with the extra term E)
     assert lw.query_variant(lw.Q5_K, 4096, 4096, 8) == lw.VARIANT_MMA
     assert lw.query_variant(lw.F16, 4096, 4096, 8) == lw.VARIANT_MMA
-    assert lw.query_variant(lw.Q6_K, 4096, 4096, 8) != lw.VARIANT_MMA
+    assert lw.query_variant(lw.Q6_K, 4096, 4096, 8) == lw.VARIANT_MMA         # q6_K: cols a multiple of 2048
+    assert lw.query_variant(lw.Q6_K, 4096, 4096 + 1024, 8) != lw.VARIANT_MMA
     assert lw.query_variant(lw.Q4_0, 4096, 4096, 1) == lw.VARIANT_IDOT        # batch 1: falls back
     lw.set_variant(lw.VARIANT_AUTO)
     assert lw.query_variant(lw.Q4_1, 4096, 4096, 16) == lw.VARIANT_MMA
