@@ -48,7 +48,7 @@ SINGLE_WORKLOADS = ("q8_0_2048",)
 DEQUANT_WORKLOADS = tuple("dequant_" + f for f in FMT_ID)
 
 
-MMA_FORMATS = ("q8_0", "q4_0", "q4_K", "q5_K", "f16", "q4_1", "q5_0", "q5_1", "q6_K")       # formats the batched tensor-core kernel takes
+MMA_FORMATS = ("q8_0", "q4_0", "q4_K", "q5_K", "f16", "q4_1", "q5_0", "q5_1", "q6_K", "q2_K")       # formats the batched tensor-core kernel takes
 
 
 def arithmetic_of(fmt, batch):

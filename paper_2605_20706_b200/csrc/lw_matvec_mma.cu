@@ -1,4 +1,4 @@
-// Batched mat-vec on the tensor cores (batch 2..16; every format but q2_K) [paper Sec 3.2: from a handful of columns on
+// Batched mat-vec on the tensor cores (batch 2..16; all ten formats) [paper Sec 3.2: from a handful of columns on
 // the mat-vec turns into a small mat-mat product, a dense contraction; Sec 3.3: one decode routine per format
 // spliced into a common skeleton].
 //
@@ -71,6 +71,8 @@ constexpr int kXPad = 64;                             // bytes after each column
 #define LW_MMA_TERMS 2
 #endif
 constexpr int kTerms = LW_MMA_TERMS;                  // terms an activation is cut into (planes in shared memory)
+constexpr int kTabRow = 72;                           // bytes between rows of a warp's scale table: 64 of entries + 8, so the
+                                                      // eight rows a warp reads at once (8-byte entries) fall into different banks
 constexpr int kSxBlockBytes = 64;                     // block sums of the activations: [block of 32][16 columns] floats
 constexpr int kMmaHeader = 128;                       // barriers, the stop flag and the grid barrier's generation
 constexpr uint32_t kGridPolls = 1u << 20;             // polls of the generation word (~0.5 us each) before giving up
@@ -193,6 +195,7 @@ struct MmaQ40 {
     static constexpr int kStageRows = 256;          // 16 warps x 16 rows
     static constexpr bool kF16 = false;
     static constexpr bool kQ6K = false;
+    static constexpr bool kQ2K = false;
     static constexpr int kPiece = 8 * 18;               // bytes of a row's 256 columns
     static constexpr bool kHasMin = false;              // no per-block offset term
     static constexpr int kTableBytes = 0;               // no per-warp table of decoded scales
@@ -224,6 +227,7 @@ struct MmaQ80 {
     static constexpr int kStageRows = 256;          // 16 warps x 16 rows
     static constexpr bool kF16 = false;
     static constexpr bool kQ6K = false;
+    static constexpr bool kQ2K = false;
     static constexpr int kPiece = 8 * 34;
     static constexpr bool kHasMin = false;
     static constexpr int kTableBytes = 0;
@@ -266,9 +270,10 @@ struct MmaQ4K {
     static constexpr int kStageRows = 256;          // 16 warps x 16 rows
     static constexpr bool kF16 = false;
     static constexpr bool kQ6K = false;
+    static constexpr bool kQ2K = false;
     static constexpr int kPiece = 144;
     static constexpr bool kHasMin = true;
-    static constexpr int kTableBytes = 16 * 8 * 8;      // per warp: 16 rows x 8 sub-blocks x (d * sc, dmin * m)
+    static constexpr int kTableBytes = 16 * kTabRow;    // per warp: 16 rows x 8 sub-blocks x (d * sc, dmin * m)
     // `rows` = address of the warp's first row piece of the stage, `tab` = the warp's table; lane: row lane / 2,
     // sub-blocks 4 (lane % 2) .. + 3
     static __device__ __forceinline__ void prepare(uint32_t rows, uint32_t tab, int lane) {
@@ -277,7 +282,7 @@ struct MmaQ4K {
         const float d = __half2float(__ushort_as_half((unsigned short)(dd & 0xFFFFu)));
         const float dmin = __half2float(__ushort_as_half((unsigned short)(dd >> 16)));
         const bool upper = lane & 1;
-        const uint32_t out = tab + (uint32_t)(lane >> 1) * 64u + (upper ? 32u : 0u);
+        const uint32_t out = tab + (uint32_t)(lane >> 1) * kTabRow + (upper ? 32u : 0u);
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             uint32_t sc, mn;
@@ -311,7 +316,7 @@ struct MmaQ4K {
     // ROW / kPiece = row of the warp's 16 (g or g + 8 is added by the caller through `tabg`): tab entry of row g
     template <int U, int BLK, int ROW>
     static __device__ __forceinline__ void scales(uint32_t, uint32_t tabg, float& d, float& m) {
-        lds_f32x2<(ROW / kPiece) * 64 + 8 * (2 * U + BLK)>(tabg, d, m);
+        lds_f32x2<(ROW / kPiece) * kTabRow + 8 * (2 * U + BLK)>(tabg, d, m);
     }
 };
 
@@ -321,6 +326,7 @@ struct MmaQ5K {
     static constexpr int kStageRows = 256;          // 16 warps x 16 rows
     static constexpr bool kF16 = false;
     static constexpr bool kQ6K = false;
+    static constexpr bool kQ2K = false;
     static constexpr int kPiece = 176;
     static constexpr bool kHasMin = true;
     static constexpr int kTableBytes = MmaQ4K::kTableBytes;
@@ -331,7 +337,7 @@ struct MmaQ5K {
         const float d = __half2float(__ushort_as_half((unsigned short)(dd & 0xFFFFu)));
         const float dmin = __half2float(__ushort_as_half((unsigned short)(dd >> 16)));
         const bool upper = lane & 1;
-        const uint32_t out = tab + (uint32_t)(lane >> 1) * 64u + (upper ? 32u : 0u);
+        const uint32_t out = tab + (uint32_t)(lane >> 1) * kTabRow + (upper ? 32u : 0u);
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             uint32_t sc, mn;
@@ -365,7 +371,7 @@ struct MmaQ5K {
     }
     template <int U, int BLK, int ROW>
     static __device__ __forceinline__ void scales(uint32_t, uint32_t tabg, float& d, float& m) {
-        lds_f32x2<(ROW / kPiece) * 64 + 8 * (2 * U + BLK)>(tabg, d, m);
+        lds_f32x2<(ROW / kPiece) * kTabRow + 8 * (2 * U + BLK)>(tabg, d, m);
     }
 };
 
@@ -384,6 +390,7 @@ struct MmaLegacy {
     static constexpr int kStageRows = 256;
     static constexpr bool kF16 = false;
     static constexpr bool kQ6K = false;
+    static constexpr bool kQ2K = false;
     static constexpr int kPiece = 8 * kBlock;
     static constexpr int kTableBytes = 0;
     static __device__ __forceinline__ void prepare(uint32_t, uint32_t, int) {}
@@ -438,6 +445,7 @@ struct MmaF16 {
     static constexpr int kStageRows = 128;
     static constexpr bool kF16 = true;
     static constexpr bool kQ6K = false;
+    static constexpr bool kQ2K = false;
     static constexpr int kPiece = 512;
     static constexpr bool kHasMin = false;
     static constexpr int kTableBytes = 0;
@@ -510,14 +518,16 @@ struct MmaQ6K {
     static constexpr int kStageRows = 256;
     static constexpr bool kF16 = false;
     static constexpr bool kQ6K = true;
+    static constexpr bool kQ2K = false;
+    static constexpr int kSuper = 210;                  // bytes of 256 weights
     static constexpr int kPiece = 224;                  // bytes fetched per row and stage (210 + up to 14 in front)
     static constexpr bool kHasMin = false;
-    static constexpr int kTableBytes = 16 * 16 * 4;     // per warp: 16 rows x 16 (d * scale)
+    static constexpr int kTableBytes = 16 * kTabRow;    // per warp: 16 rows x 16 (d * scale)
     // rows = the warp's first row piece + o; lane: row lane / 2, scales 8 (lane % 2) .. + 7
     static __device__ __forceinline__ void prepare(uint32_t rows, uint32_t tab, int lane) {
         const uint32_t row = rows + (uint32_t)(lane >> 1) * kPiece;
         const float d = lds_half<208>(row);
-        const uint32_t sc = row + 192u + 8u * (lane & 1), out = tab + (uint32_t)(lane >> 1) * 64u + 32u * (lane & 1);
+        const uint32_t sc = row + 192u + 8u * (lane & 1), out = tab + (uint32_t)(lane >> 1) * kTabRow + 32u * (lane & 1);
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
             int v;
@@ -526,6 +536,100 @@ struct MmaQ6K {
         }
     }
 };
+
+// q2_K: 84-byte super-blocks {16 bytes of 4-bit scale | 4-bit offset (one per 16 weights), 64 bytes of 2-bit codes, d,
+// dmin}: weight = d * sc * q - dmin * m.  84 is a multiple of 4 but not of 16: fetched like q6_K from the 16-byte
+// boundary below the piece (96 bytes per row), the remainder is a whole number of words.  Group j (0..3) of a half
+// of 128 weights is bits 2j, 2j+1 of the half's 32 bytes.  Codes 0..3 are exact in bf16; the offsets go onto fp32
+// sums of each 16 activations (extra term E, c = 2^-18).  Unit U = half U / 2, groups {0, 1} or {2, 3}.
+struct MmaQ2K {
+    static constexpr int kStageRows = 256;
+    static constexpr bool kF16 = false;
+    static constexpr bool kQ6K = false;
+    static constexpr bool kQ2K = true;
+    static constexpr int kSuper = 84;
+    static constexpr int kPiece = 96;
+    static constexpr bool kHasMin = false;              // (its own block step applies the offsets)
+    static constexpr int kTabRow2 = 136;                // 128 bytes of entries + 8 (bank spread as above)
+    static constexpr int kTableBytes = 16 * kTabRow2;   // per warp: 16 rows x 16 x (d * sc, dmin * m)
+    // rows = the warp's first row piece + o; lane: row lane / 2, sub-blocks 8 (lane % 2) .. + 7
+    static __device__ __forceinline__ void prepare(uint32_t rows, uint32_t tab, int lane) {
+        const uint32_t row = rows + (uint32_t)(lane >> 1) * kPiece;
+        const uint32_t dd = lds32<80>(row);
+        const float d = __half2float(__ushort_as_half((unsigned short)(dd & 0xFFFFu)));
+        const float dmin = __half2float(__ushort_as_half((unsigned short)(dd >> 16)));
+        const uint32_t w0 = lds32<0>(row + 8u * (lane & 1)), w1 = lds32<4>(row + 8u * (lane & 1));
+        const uint32_t out = tab + (uint32_t)(lane >> 1) * kTabRow2 + 64u * (lane & 1);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const uint32_t b = ((j < 4 ? w0 : w1) >> (8 * (j & 3))) & 0xFFu;
+            asm volatile("st.shared.v2.f32 [%0], {%1, %2};" ::"r"(out + 8u * j), "f"(d * (float)(b & 0xFu)),
+                         "f"(dmin * (float)(b >> 4))
+                         : "memory");
+        }
+    }
+};
+
+// One group of 32 q2_K weights of the warp's 16 rows against all columns.  tabg = the warp's table at row g; sx = the
+// lane's sums of 16 activations: [block of 32][half][16 columns], columns 2 t and 2 t + 1, group nt 32 bytes further.
+template <int NT, int U, int BLK>
+__device__ __forceinline__ void block_step_q2k(uint32_t wt, uint32_t tabg, uint32_t sx, const uint32_t (&xp)[NT][kTerms],
+                                               float (&y)[NT][4]) {
+    constexpr int kHalf = U / 2, kGroup = 2 * (U & 1) + BLK, kShift = 2 * kGroup;
+    constexpr int kQs = 16 + 32 * kHalf, kRow8 = 8 * MmaQ2K::kPiece;
+    const uint32_t bias = 0x43004300u;                  // (128 + q) - 128 = q, exactly
+    uint32_t a[4], b[4];
+    {
+        const uint32_t q0 = (lds32<kQs>(wt) >> kShift) & 0x03030303u, q1 = (lds32<kQs + 16>(wt) >> kShift) & 0x03030303u;
+        a[0] = sub_bf16x2(bytes_to_bf16_128_plus<0>(q0), bias);
+        a[1] = sub_bf16x2(bytes_to_bf16_128_plus<2>(q0), bias);
+        a[2] = sub_bf16x2(bytes_to_bf16_128_plus<0>(q1), bias);
+        a[3] = sub_bf16x2(bytes_to_bf16_128_plus<2>(q1), bias);
+        const uint32_t r0 = (lds32<kRow8 + kQs>(wt) >> kShift) & 0x03030303u,
+                       r1 = (lds32<kRow8 + kQs + 16>(wt) >> kShift) & 0x03030303u;
+        b[0] = sub_bf16x2(bytes_to_bf16_128_plus<0>(r0), bias);
+        b[1] = sub_bf16x2(bytes_to_bf16_128_plus<2>(r0), bias);
+        b[2] = sub_bf16x2(bytes_to_bf16_128_plus<0>(r1), bias);
+        b[3] = sub_bf16x2(bytes_to_bf16_128_plus<2>(r1), bias);
+    }
+    // (d * sc, dmin * m) of the group's two halves: row g, then row g + 8
+    float d00, m00, d01, m01, d10, m10, d11, m11;
+    constexpr int kT = 8 * (8 * kHalf + 2 * kGroup);
+    lds_f32x2<kT>(tabg, d00, m00);
+    lds_f32x2<kT + 8>(tabg, d01, m01);
+    lds_f32x2<8 * MmaQ2K::kTabRow2 + kT>(tabg, d10, m10);
+    lds_f32x2<8 * MmaQ2K::kTabRow2 + kT + 8>(tabg, d11, m11);
+    constexpr int kX = 2 * (64 * U + 32 * BLK);
+    constexpr int kS = 128 * (2 * U + BLK);              // the block's sums of activations
+#pragma unroll
+    for (int nt = 0; nt < NT; ++nt) {
+        float c0[4], c1[4];
+#pragma unroll
+        for (int s = 0; s < kTerms; ++s) {
+            uint32_t b0, b1, b2, b3;
+            lds128<kX>(xp[nt][s], b0, b1, b2, b3);
+            if (s == 0) {
+                mma_bf16_first(c0, a[0], b[0], a[1], b[1], b0, b1);
+                mma_bf16_first(c1, a[2], b[2], a[3], b[3], b2, b3);
+            } else {
+                mma_bf16(c0, a[0], b[0], a[1], b[1], b0, b1);
+                mma_bf16(c1, a[2], b[2], a[3], b[3], b2, b3);
+            }
+        }
+        float s00, s01, s10, s11;                        // sums of the first / second 16 activations, columns 2t, 2t+1
+        if (nt == 0) {
+            lds_f32x2<kS>(sx, s00, s01);
+            lds_f32x2<kS + 64>(sx, s10, s11);
+        } else {
+            lds_f32x2<kS + 32>(sx, s00, s01);
+            lds_f32x2<kS + 64 + 32>(sx, s10, s11);
+        }
+        y[nt][0] = fmaf(-m01, s10, fmaf(-m00, s00, fmaf(d01, c1[0], fmaf(d00, c0[0], y[nt][0]))));
+        y[nt][1] = fmaf(-m01, s11, fmaf(-m00, s01, fmaf(d01, c1[1], fmaf(d00, c0[1], y[nt][1]))));
+        y[nt][2] = fmaf(-m11, s10, fmaf(-m10, s00, fmaf(d11, c1[2], fmaf(d10, c0[2], y[nt][2]))));
+        y[nt][3] = fmaf(-m11, s11, fmaf(-m10, s01, fmaf(d11, c1[3], fmaf(d10, c0[3], y[nt][3]))));
+    }
+}
 
 // A 32-bit word of the piece at byte OFF from `wt` (word-aligned address below the piece's word + 4 t); MIS: the piece
 // is two bytes off the word grid.
@@ -567,7 +671,7 @@ __device__ __forceinline__ void block_step_q6k(uint32_t wt, uint32_t tabg, const
     }
     float s00, s01, s10, s11;                            // d * scale of (row g, half 0 / 1), (row g + 8, half 0 / 1)
     lds_f32x2<4 * (8 * kHalf + 2 * kGroup)>(tabg, s00, s01);
-    lds_f32x2<8 * 64 + 4 * (8 * kHalf + 2 * kGroup)>(tabg, s10, s11);
+    lds_f32x2<8 * kTabRow + 4 * (8 * kHalf + 2 * kGroup)>(tabg, s10, s11);
     constexpr int kX = 2 * (64 * U + 32 * BLK);
 #pragma unroll
     for (int nt = 0; nt < NT; ++nt) {
@@ -800,11 +904,11 @@ __global__ void __launch_bounds__(kMmaThreads, kCtasPerSm) matvec_mma_kernel(con
                     tensor_load_2d(smem + p.w_off + (size_t)cur.slot * kStageBytes + u * MmaF16::kSliceBytes,
                                    &maps.m[cur.it], ((cur.c * spc + cur.j) * 4 + u) * 32,
                                    (cur.rs - p.item[cur.it].rs_begin) * kStageRows, &full[cur.slot], policy);
-            } else if constexpr (T::kQ6K) {
-                // the piece starts at byte 210 * (stage's column index) of the row: fetch from the 16-byte boundary below
+            } else if constexpr (T::kQ6K || T::kQ2K) {
+                // the piece starts at byte kSuper * (stage's column index) of the row: fetch from the 16-byte boundary below
                 tensor_load_2d(smem + p.w_off + (size_t)cur.slot * kStageBytes, &maps.m[cur.it],
-                               ((210 * (cur.c * spc + cur.j)) >> 4) << 2, (cur.rs - p.item[cur.it].rs_begin) * kStageRows,
-                               &full[cur.slot], policy);
+                               ((T::kSuper * (cur.c * spc + cur.j)) >> 4) << 2,
+                               (cur.rs - p.item[cur.it].rs_begin) * kStageRows, &full[cur.slot], policy);
             } else {
                 tensor_load_2d(smem + p.w_off + (size_t)cur.slot * kStageBytes, &maps.m[cur.it],
                                (cur.c * spc + cur.j) * (kPiece / 4), (cur.rs - p.item[cur.it].rs_begin) * kStageRows,
@@ -968,6 +1072,14 @@ __global__ void __launch_bounds__(kMmaThreads, kCtasPerSm) matvec_mma_kernel(con
                             split3(v[q][nt].z, h[0][2], h[1][2], h[2][2]);
                             split3(v[q][nt].w, h[0][3], h[1][3], h[2][3]);
                         }
+                        if constexpr (T::kQ2K) {
+                            // sums of each 16 activations (four consecutive lanes hold them): [block][half][column]
+                            float sum = (v[q][nt].x + v[q][nt].y) + (v[q][nt].z + v[q][nt].w);
+                            sum += __shfl_xor_sync(0xffffffffu, sum, 1);
+                            sum += __shfl_xor_sync(0xffffffffu, sum, 2);
+                            if ((lane & 3) == 0)
+                                *reinterpret_cast<float*>(smem + p.sx_off + (size_t)(k4 >> 3) * 128 + ((k4 >> 2) & 1) * 64 + 4 * b) = sum;
+                        }
                         if constexpr (T::kHasMin) {
                             // sum of each block of 32 activations (eight consecutive lanes hold one), for the
                             // formats with a per-block offset: [block of the chunk][column]
@@ -999,10 +1111,10 @@ __global__ void __launch_bounds__(kMmaThreads, kCtasPerSm) matvec_mma_kernel(con
         const int64_t r0 = (int64_t)(rs - mat.rs_begin) * kStageRows;
         if (r0 + 16 * mt < mat.rows) {
             const uint32_t row = wrow + (uint32_t)slot * kStageBytes, wt = row + 4u * t;
-            const uint32_t tab = smem_u32(smem + p.tab_off) + (uint32_t)warp * T::kTableBytes, tabg = tab + 64u * g;
+            const uint32_t tab = smem_u32(smem + p.tab_off) + (uint32_t)warp * T::kTableBytes, tabg = tab + (uint32_t)kTabRow * g;
             const uint32_t sx = smem_u32(smem + p.sx_off) + (uint32_t)(8 * j) * kSxBlockBytes + 8u * t;
-            if constexpr (T::kQ6K) {
-                const uint32_t o = (uint32_t)(210 * (c * spc + j)) & 15u;      // the piece's offset in the fetched bytes
+            if constexpr (T::kQ6K || T::kQ2K) {
+                const uint32_t o = (uint32_t)(T::kSuper * (c * spc + j)) & 15u;      // the piece's offset in the fetched bytes
                 T::prepare(row - (uint32_t)g * kPiece + o, tab, lane);
                 __syncwarp();
             } else if constexpr (T::kTableBytes > 0) {
@@ -1015,7 +1127,18 @@ __global__ void __launch_bounds__(kMmaThreads, kCtasPerSm) matvec_mma_kernel(con
 #pragma unroll
                 for (int s = 0; s < kTerms; ++s)
                     xp[nt][s] = xlane + 2u * (uint32_t)(j * kStageCols) + s * plane_pitch + nt * 8 * x_pitch;
-            if constexpr (T::kQ6K) {
+            if constexpr (T::kQ2K) {
+                const uint32_t wo = wt + ((uint32_t)(84 * (c * spc + j)) & 15u);
+                const uint32_t tq = tab + (uint32_t)MmaQ2K::kTabRow2 * g, sq = smem_u32(smem + p.sx_off) + (uint32_t)(8 * j) * 128u + 8u * t;
+                block_step_q2k<NT, 0, 0>(wo, tq, sq, xp, y);
+                block_step_q2k<NT, 0, 1>(wo, tq, sq, xp, y);
+                block_step_q2k<NT, 1, 0>(wo, tq, sq, xp, y);
+                block_step_q2k<NT, 1, 1>(wo, tq, sq, xp, y);
+                block_step_q2k<NT, 2, 0>(wo, tq, sq, xp, y);
+                block_step_q2k<NT, 2, 1>(wo, tq, sq, xp, y);
+                block_step_q2k<NT, 3, 0>(wo, tq, sq, xp, y);
+                block_step_q2k<NT, 3, 1>(wo, tq, sq, xp, y);
+            } else if constexpr (T::kQ6K) {
                 const uint32_t o = (uint32_t)(210 * (c * spc + j)) & 15u;
                 if (o & 2u)
                     stage_q6k<NT, true>(wt + (o & ~3u), tabg, xp, y);
@@ -1134,10 +1257,12 @@ bool mma_plan(int fmt, int64_t cols, int nt, int& chunk_cols, int& ring, size_t&
                       : fmt == LW_Q5_0 ? MmaLegacy<LW_Q5_0>::kPiece
                       : fmt == LW_Q5_1 ? MmaLegacy<LW_Q5_1>::kPiece
                       : fmt == LW_Q6_K ? MmaQ6K::kPiece
+                      : fmt == LW_Q2_K ? MmaQ2K::kPiece
                                        : MmaF16::kPiece;
     stage_bytes = (size_t)mma_stage_rows(fmt) * piece;
     // q4_K: block sums of the activations (64 bytes per block of a chunk of up to 1024 columns) and the warps' tables
-    extra_bytes = (fmt == LW_Q4_K || fmt == LW_Q5_K || fmt == LW_Q6_K)
+    extra_bytes = fmt == LW_Q2_K ? (size_t)(1024 / 32) * 128 + (size_t)kMmaWarps * MmaQ2K::kTableBytes
+                  : (fmt == LW_Q4_K || fmt == LW_Q5_K || fmt == LW_Q6_K)
                       ? (size_t)(1024 / 32) * kSxBlockBytes + (size_t)kMmaWarps * MmaQ4K::kTableBytes
                       : ((fmt == LW_F16 || fmt == LW_Q4_1 || fmt == LW_Q5_1) ? (size_t)(1024 / 32) * kSxBlockBytes : 0);
     // (f16: up to 1 KB more goes into aligning the swizzled stages)
@@ -1160,9 +1285,10 @@ bool mma_plan(int fmt, int64_t cols, int nt, int& chunk_cols, int& ring, size_t&
 
 bool matvec_mma_supported(int fmt, int64_t rows, int64_t cols, int batch) {
     if (fmt != LW_Q4_0 && fmt != LW_Q8_0 && fmt != LW_Q4_K && fmt != LW_Q5_K && fmt != LW_F16 && fmt != LW_Q4_1 &&
-        fmt != LW_Q5_0 && fmt != LW_Q5_1 && fmt != LW_Q6_K)
+        fmt != LW_Q5_0 && fmt != LW_Q5_1 && fmt != LW_Q6_K && fmt != LW_Q2_K)
         return false;
     if (fmt == LW_Q6_K && cols % 2048 != 0) return false;      // 210-byte super-blocks: rows must be whole 16-byte units
+    if (fmt == LW_Q2_K && cols % 1024 != 0) return false;      // 84-byte super-blocks likewise
     if (batch < 2 || batch > 16) return false;
     if (cols % kStageCols != 0) return false;
     return rows >= 1 && rows <= (int64_t)1 << 30;
@@ -1251,7 +1377,8 @@ int launch_matvec_mma_group(int fmt, int64_t cols, int n_items, const void* cons
     p.grid_bar = grid_bar;
     p.x_off = kMmaHeader;
     p.sx_off = (uint32_t)(kMmaHeader + x_bytes);
-    p.tab_off = p.sx_off + (uint32_t)((fmt == LW_Q4_K || fmt == LW_Q5_K || fmt == LW_Q6_K) ? (1024 / 32) * kSxBlockBytes : 0);
+    p.tab_off = p.sx_off + (uint32_t)(fmt == LW_Q2_K ? (1024 / 32) * 128
+                                      : (fmt == LW_Q4_K || fmt == LW_Q5_K || fmt == LW_Q6_K) ? (1024 / 32) * kSxBlockBytes : 0);
     // the stages: 128-byte aligned; f16's swizzle pattern is one of address bits, so its stages start on 1 KB
     const size_t w_align = fmt == LW_F16 ? 1024 : 128;
     p.w_off = (uint32_t)((kMmaHeader + x_bytes + extra_bytes + w_align - 1) / w_align * w_align);
@@ -1280,6 +1407,9 @@ int launch_matvec_mma_group(int fmt, int64_t cols, int n_items, const void* cons
     if (fmt == LW_F16)
         return nt == 1 ? launch_mma<MmaF16, 1>(p, maps, grid, smem_bytes, overlap != 0, stream)
                        : launch_mma<MmaF16, 2>(p, maps, grid, smem_bytes, overlap != 0, stream);
+    if (fmt == LW_Q2_K)
+        return nt == 1 ? launch_mma<MmaQ2K, 1>(p, maps, grid, smem_bytes, overlap != 0, stream)
+                       : launch_mma<MmaQ2K, 2>(p, maps, grid, smem_bytes, overlap != 0, stream);
     if (fmt == LW_Q6_K)
         return nt == 1 ? launch_mma<MmaQ6K, 1>(p, maps, grid, smem_bytes, overlap != 0, stream)
                        : launch_mma<MmaQ6K, 2>(p, maps, grid, smem_bytes, overlap != 0, stream);

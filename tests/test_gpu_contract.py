@@ -132,7 +132,7 @@ def test_batched_kernels_need_no_extra_term(fmt, kernel):
 
 
 @pytest.mark.parametrize("fmt,c_extra", [(lw.Q4_K, 2.0 ** -18), (lw.Q5_K, 2.0 ** -18), (lw.F16, 2.0 ** -30),
-                                         (lw.Q4_1, 2.0 ** -18), (lw.Q5_1, 2.0 ** -18)])
+                                         (lw.Q4_1, 2.0 ** -18), (lw.Q5_1, 2.0 ** -18), (lw.Q2_K, 2.0 ** -18)])
 def test_formats_with_an_extra_term_on_the_tensor_cores_stay_inside_the_stated_bound(fmt, c_extra):
     # q4_K / q5_K in the batched tensor-core kernel apply the sub-block offsets to sums of activations, like the
     # fp32-activation streaming family: the header gives them the extra term with c = 2^-18; f16 holds the

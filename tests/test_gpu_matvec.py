@@ -100,12 +100,14 @@ def test_matvec_mma_kernel(fmt, batch, rows, cols):
 
 
 @pytest.mark.parametrize("batch", [3, 8, 13, 16])
-@pytest.mark.parametrize("rows,cols", [(1, 2048), (17, 2048), (255, 4096), (300, 6144), (513, 14336), (4096, 2048)])
-def test_matvec_mma_kernel_q6_K(batch, rows, cols):
-    # q6_K on the tensor cores: 210-byte super-blocks, so a stage's row pieces start on a 2-byte grid inside the
-    # 16-byte-aligned fetch (all eight remainders occur from 16 column stages on, the odd ones with straddled
-    # words); cols must be a multiple of 2048
-    fmt = lw.Q6_K
+@pytest.mark.parametrize("fmt,rows,cols", [(lw.Q6_K, 1, 2048), (lw.Q6_K, 17, 2048), (lw.Q6_K, 255, 4096), (lw.Q6_K, 300, 6144),
+                                           (lw.Q6_K, 513, 14336), (lw.Q6_K, 4096, 2048), (lw.Q2_K, 1, 1024),
+                                           (lw.Q2_K, 17, 3072), (lw.Q2_K, 255, 4096), (lw.Q2_K, 513, 14336),
+                                           (lw.Q2_K, 4096, 2048)])
+def test_matvec_mma_kernel_offset_fetch(fmt, batch, rows, cols):
+    # q6_K and q2_K on the tensor cores: 210- and 84-byte super-blocks, so a stage's row pieces start on a 2-byte
+    # (4-byte) grid inside the 16-byte-aligned fetch; all remainders occur from 16 (4) column stages on, q6_K's odd
+    # ones with straddled words; cols must be a multiple of 2048 (1024)
     lw.set_variant(lw.VARIANT_AUTO)
     assert lw.query_variant(fmt, rows, cols, batch) == lw.VARIANT_MMA
     assert lw.query_variant(fmt, rows, cols + 256, batch) != lw.VARIANT_MMA
@@ -113,7 +115,7 @@ def test_matvec_mma_kernel_q6_K(batch, rows, cols):
     X = synth.activations(66, batch, batch, cols)
     y_ref, s_ref = oracle.matvec(fmt, blocks, rows, cols, X, batch, nthreads=8)
     y = gpu_matvec(fmt, blocks, rows, cols, X, batch, lw.VARIANT_AUTO)
-    check_matvec(y, y_ref, s_ref, "mma q6_K %dx%d batch %d" % (rows, cols, batch))
+    check_matvec(y, y_ref, s_ref, "mma fmt %d %dx%d batch %d" % (fmt, rows, cols, batch))
     # and two matrices in one launch
     w = torch.from_numpy(blocks).cuda()
     x = torch.from_numpy(X).cuda()
@@ -122,7 +124,7 @@ def test_matvec_mma_kernel_q6_K(batch, rows, cols):
     torch.cuda.synchronize()
     for yg in ys:
         yg.check("grouped Y")
-        check_matvec(yg.t.cpu().numpy(), y_ref, s_ref, "grouped mma q6_K")
+        check_matvec(yg.t.cpu().numpy(), y_ref, s_ref, "grouped mma fmt %d" % fmt)
     assert lw.device_status() == 0
 
 

@@ -149,7 +149,8 @@ def test_variant_controls():
     assert lw.query_variant(lw.Q4_0, 4096, 4096, 1) == lw.VARIANT_IDOT        # batch 1: falls back
     lw.set_variant(lw.VARIANT_AUTO)
     assert lw.query_variant(lw.Q4_1, 4096, 4096, 16) == lw.VARIANT_MMA
-    assert lw.query_variant(lw.Q2_K, 4096, 4096, 16) == lw.VARIANT_IDOT      # no tensor-core form: one pass per column
+    assert lw.query_variant(lw.Q2_K, 4096, 4096, 16) == lw.VARIANT_MMA       # q2_K: cols a multiple of 1024
+    assert lw.query_variant(lw.Q2_K, 4096, 4096 + 512, 16) == lw.VARIANT_GENERIC   # rows not whole 16-byte pieces
     assert lw.query_variant(lw.Q8_0, 16, 96, 3) == lw.VARIANT_GENERIC       # cols % 256 != 0: tiled fp32 kernel
     assert lw.query_variant(lw.Q6_K, 4096, 4096, 1) == lw.VARIANT_IDOT
     assert lw.query_variant(lw.Q5_K, 4096, 4096, 1) == lw.VARIANT_IDOT
