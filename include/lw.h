@@ -103,7 +103,7 @@ int lw_dequant(int fmt, const void* W_blocks, int64_t n, float* out, void* strea
 
 /* Fused dequantise + mat-vec [Sec 3.2, 3.3]: Y[b*rows + r] = sum_k decode(W)[r][k] * X[b*cols + k],
  * fp32 accumulation, for b < batch (1..16).  The batched kernels reuse every decoded block for all
- * their columns: without a forced variant every format but q2_K, with cols a multiple of 256 (q6_K: of 2048), runs on the tensor
+ * their columns: without a forced variant every format, with cols a multiple of 256 (q6_K: of 2048, q2_K: of 1024), runs on the tensor
  * cores from three columns on (LW_VARIANT_MMA); the other quantised formats (and f16 up to four columns)
  * run one streaming pass per column instead (four columns per launch), which measures faster on B200
  * than their batched kernels.
@@ -122,7 +122,7 @@ int lw_dequant(int fmt, const void* W_blocks, int64_t n, float* out, void* strea
  * (23 bits + sign relative to the largest magnitude in each run of 16 or 32), so an activation that is
  * huge compared with its neighbours and meets a weight that is zero or nearly so leaves an absolute error
  * that S does not cover.  For them
- *     E = c * sum_k What_k * A_k ,   c = 2^-18 (IDOT, the default for the quantised formats; MMA on q4_K / q5_K / q4_1 / q5_1), 2^-16 (STREAM),
+ *     E = c * sum_k What_k * A_k ,   c = 2^-18 (IDOT, the default for the quantised formats; MMA on q4_K / q5_K / q2_K / q4_1 / q5_1), 2^-16 (STREAM),
  *                                    2^-30 (MMA on f16: activations as two f16 terms relative to their block's largest),
  * where, over the aligned run of 32 columns that contains k, A_k is the largest |x| and What_k the largest
  * decoded |w|.  This holds for weights made by lw_quantize, and for any block whose scale * code and offset
@@ -158,7 +158,7 @@ typedef struct {
 int lw_matvec_group(int fmt, int64_t cols, int n_items, const lw_group_item* items, void* stream);
 
 /* The same with `batch` activation columns per item (1..16): X of an item is batch * cols floats, Y batch * rows
- * floats, laid out as in lw_matvec.  batch 1 is lw_matvec_group.  From two columns on, every format but q2_K with cols a
+ * floats, laid out as in lw_matvec.  batch 1 is lw_matvec_group.  From two columns on, every format with cols a
  * multiple of 256 run all items in ONE launch of the tensor-core kernel (LW_VARIANT_MMA, unless another variant
  * is forced; items that follow one another and share their X pointer share its converted copy); everything else
  * is run item by item with lw_matvec.  Errors as lw_matvec (LW_ERR_BATCH for batch outside 1..16); a call that
@@ -243,7 +243,7 @@ typedef enum {
                                block's sum; every fp32 activation is cut into two bf16 terms that add up to it within
                                2^-16 of its magnitude (an error that scales with |w x| term by term and stays at
                                0.15 of the tolerance at worst), so E = 0 in the accuracy statement of lw_matvec for
-                               q8_0, q4_0, q5_0 and q6_K (cols a multiple of 2048).  q4_K, q5_K, q4_1 and q5_1 as well: there the codes are
+                               q8_0, q4_0, q5_0 and q6_K (cols a multiple of 2048).  q4_K, q5_K, q2_K (cols a multiple of 1024), q4_1 and q5_1 as well: there the codes are
                                multiplied the same way, and the sub-block offsets
                                (dmin * m) are applied to fp32 sums of each sub-block's activations, which brings the
                                extra term E back with c = 2^-18.  cols a multiple of 256; all columns in one pass

@@ -49,7 +49,7 @@ bool matvec_tile_supported(int fmt, int64_t rows, int64_t cols, int batch);
 int launch_matvec_tile(int fmt, const void* W, int64_t rows, int64_t cols, const float* X, float* Y, int batch,
                        cudaStream_t stream);
 // Batched tensor-core kernel (2..16 columns; weights as exact bf16 codes, activations as three bf16 terms, fp32
-// accumulation; f16: f16 operands): every format but q2_K, cols a multiple of 256 (q6_K: of 2048).  The launch clears Y first (the kernel adds into it).
+// accumulation; f16: f16 operands): every format, cols a multiple of 256 (q6_K: of 2048, q2_K: of 1024).  The launch clears Y first (the kernel adds into it).
 bool matvec_mma_supported(int fmt, int64_t rows, int64_t cols, int batch);
 int launch_matvec_mma(int fmt, const void* W, int64_t rows, int64_t cols, const float* X, float* Y, int batch,
                       int overlap, bool self_clear, cudaStream_t stream);

@@ -84,7 +84,7 @@ def test_matvec_tile_kernel(fmt, batch, rows, cols):
 @pytest.mark.parametrize("rows,cols", [(1, 256), (15, 512), (16, 1024), (17, 768), (255, 2048), (256, 1024), (257, 4096),
                                        (333, 3072), (1000, 14336), (4096, 1280), (70000, 1024)])
 def test_matvec_mma_kernel(fmt, batch, rows, cols):
-    # the batched tensor-core kernel (AUTO's choice for every format but q2_K (q6_K: its own test) from three columns on when cols is a
+    # the batched tensor-core kernel (AUTO's choice for every format (q6_K and q2_K: their own test) from three columns on when cols is a
     # multiple of 256): ragged row counts around its 16-row fragments and 256-row stages, chunks of 256 / 512 / 1024 columns,
     # one and two groups of eight columns, more stages than CTAs (70000 rows) and fewer (1 row)
     lw.set_variant(lw.VARIANT_AUTO)
