@@ -197,6 +197,7 @@ struct MmaQ40 {
     static constexpr bool kQ6K = false;
     static constexpr bool kQ2K = false;
     static constexpr int kPiece = 8 * 18;               // bytes of a row's 256 columns
+    static constexpr int kXWords = kPiece / 4;          // 32-bit words between consecutive stages of a row
     static constexpr bool kHasMin = false;              // no per-block offset term
     static constexpr int kTableBytes = 0;               // no per-warp table of decoded scales
     static __device__ __forceinline__ void prepare(uint32_t, uint32_t, int) {}
@@ -229,6 +230,7 @@ struct MmaQ80 {
     static constexpr bool kQ6K = false;
     static constexpr bool kQ2K = false;
     static constexpr int kPiece = 8 * 34;
+    static constexpr int kXWords = kPiece / 4;
     static constexpr bool kHasMin = false;
     static constexpr int kTableBytes = 0;
     static __device__ __forceinline__ void prepare(uint32_t, uint32_t, int) {}
@@ -272,6 +274,7 @@ struct MmaQ4K {
     static constexpr bool kQ6K = false;
     static constexpr bool kQ2K = false;
     static constexpr int kPiece = 144;
+    static constexpr int kXWords = kPiece / 4;
     static constexpr bool kHasMin = true;
     static constexpr int kTableBytes = 16 * kTabRow;    // per warp: 16 rows x 8 sub-blocks x (d * sc, dmin * m)
     // `rows` = address of the warp's first row piece of the stage, `tab` = the warp's table; lane: row lane / 2,
@@ -328,6 +331,7 @@ struct MmaQ5K {
     static constexpr bool kQ6K = false;
     static constexpr bool kQ2K = false;
     static constexpr int kPiece = 176;
+    static constexpr int kXWords = kPiece / 4;
     static constexpr bool kHasMin = true;
     static constexpr int kTableBytes = MmaQ4K::kTableBytes;
     static __device__ __forceinline__ void prepare(uint32_t rows, uint32_t tab, int lane) {
@@ -391,7 +395,10 @@ struct MmaLegacy {
     static constexpr bool kF16 = false;
     static constexpr bool kQ6K = false;
     static constexpr bool kQ2K = false;
-    static constexpr int kPiece = 8 * kBlock;
+    // 16 bytes more than a row's 256 columns are fetched for q4_1 and q5_1: their 160- and 192-byte pitches would put
+    // the eight rows a warp reads at once into four resp. two banks (176 and 208 spread them over eight)
+    static constexpr int kPiece = 8 * kBlock + (FMT == LW_Q5_0 ? 0 : 16);
+    static constexpr int kXWords = 8 * kBlock / 4;
     static constexpr int kTableBytes = 0;
     static __device__ __forceinline__ void prepare(uint32_t, uint32_t, int) {}
     // wt = the row's piece + 4 t, row = the row's piece, t = lane % 4
@@ -508,7 +515,7 @@ __device__ __forceinline__ void block_step_f16(uint32_t wrow, const uint32_t (&s
 
 // q6_K: 210-byte super-blocks {128 bytes of low nibbles, 64 bytes of upper bit pairs, 16 int8 scales (one per 16
 // weights), d}.  210 is not a multiple of 16, so a row's piece of a stage starts anywhere on a 2-byte grid: the
-// tensor copy starts at the 16-byte boundary below it and fetches 224 bytes per row, and the kernel indexes from
+// tensor copy starts at the 16-byte boundary below it and fetches 240 bytes per row, and the kernel indexes from
 // the remainder `o` (0, 2, .. 14); where o is 2 modulo 4 every word of the piece straddles two words of shared
 // memory (MIS: two loads and a byte permute).  A code is nibble | two upper bits << 4 = 0..63, minus 32: exact in
 // bf16, and there is no offset term: E = 0.  The two 16-weight halves of a block have their own scales, so the two
@@ -520,7 +527,8 @@ struct MmaQ6K {
     static constexpr bool kQ6K = true;
     static constexpr bool kQ2K = false;
     static constexpr int kSuper = 210;                  // bytes of 256 weights
-    static constexpr int kPiece = 224;                  // bytes fetched per row and stage (210 + up to 14 in front)
+    static constexpr int kPiece = 240;                  // bytes fetched per row and stage: 210 + up to 14 in front, and 16
+                                                        // more so that the pitch spreads eight rows over eight banks
     static constexpr bool kHasMin = false;
     static constexpr int kTableBytes = 16 * kTabRow;    // per warp: 16 rows x 16 (d * scale)
     // rows = the warp's first row piece + o; lane: row lane / 2, scales 8 (lane % 2) .. + 7
@@ -539,7 +547,7 @@ struct MmaQ6K {
 
 // q2_K: 84-byte super-blocks {16 bytes of 4-bit scale | 4-bit offset (one per 16 weights), 64 bytes of 2-bit codes, d,
 // dmin}: weight = d * sc * q - dmin * m.  84 is a multiple of 4 but not of 16: fetched like q6_K from the 16-byte
-// boundary below the piece (96 bytes per row), the remainder is a whole number of words.  Group j (0..3) of a half
+// boundary below the piece (112 bytes per row), the remainder is a whole number of words.  Group j (0..3) of a half
 // of 128 weights is bits 2j, 2j+1 of the half's 32 bytes.  Codes 0..3 are exact in bf16; the offsets go onto fp32
 // sums of each 16 activations (extra term E, c = 2^-18).  Unit U = half U / 2, groups {0, 1} or {2, 3}.
 struct MmaQ2K {
@@ -548,7 +556,7 @@ struct MmaQ2K {
     static constexpr bool kQ6K = false;
     static constexpr bool kQ2K = true;
     static constexpr int kSuper = 84;
-    static constexpr int kPiece = 96;
+    static constexpr int kPiece = 112;                  // 84 + up to 12 in front + 16 (bank spread, as for q6_K)
     static constexpr bool kHasMin = false;              // (its own block step applies the offsets)
     static constexpr int kTabRow2 = 136;                // 128 bytes of entries + 8 (bank spread as above)
     static constexpr int kTableBytes = 16 * kTabRow2;   // per warp: 16 rows x 16 x (d * sc, dmin * m)
@@ -911,7 +919,7 @@ __global__ void __launch_bounds__(kMmaThreads, kCtasPerSm) matvec_mma_kernel(con
                                (cur.rs - p.item[cur.it].rs_begin) * kStageRows, &full[cur.slot], policy);
             } else {
                 tensor_load_2d(smem + p.w_off + (size_t)cur.slot * kStageBytes, &maps.m[cur.it],
-                               (cur.c * spc + cur.j) * (kPiece / 4), (cur.rs - p.item[cur.it].rs_begin) * kStageRows,
+                               (cur.c * spc + cur.j) * T::kXWords, (cur.rs - p.item[cur.it].rs_begin) * kStageRows,
                                &full[cur.slot], policy);
             }
         }
