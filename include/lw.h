@@ -103,10 +103,10 @@ int lw_dequant(int fmt, const void* W_blocks, int64_t n, float* out, void* strea
 
 /* Fused dequantise + mat-vec [Sec 3.2, 3.3]: Y[b*rows + r] = sum_k decode(W)[r][k] * X[b*cols + k],
  * fp32 accumulation, for b < batch (1..16).  The batched kernels reuse every decoded block for all
- * their columns: without a forced variant every format, with cols a multiple of 256 (q6_K: of 2048, q2_K: of 1024), runs on the tensor
- * cores from three columns on (LW_VARIANT_MMA); the other quantised formats (and f16 up to four columns)
- * run one streaming pass per column instead (four columns per launch), which measures faster on B200
- * than their batched kernels.
+ * their columns: without a forced variant every format, with cols a multiple of 256 (q6_K: of 2048,
+ * q2_K: of 1024), runs on the tensor cores from three columns on (LW_VARIANT_MMA); two columns, and other
+ * widths of the streaming shapes, run one streaming pass per column instead (four columns per launch), which
+ * measures faster on B200 than the older batched kernels.
  * W_blocks: device, rows * lw_row_bytes(fmt, cols) bytes, row-major without padding, 16-byte
  *           aligned, read-only.
  * X: device, batch * cols floats, each activation vector contiguous, 16-byte aligned, read-only.
@@ -115,15 +115,17 @@ int lw_dequant(int fmt, const void* W_blocks, int64_t n, float* out, void* strea
  * Accuracy.  With w the decoded weights and S = sum_k |w_k x_k|, every result satisfies
  *     |y - y_exact| <= 1e-4 * S + 1e-6 + E .
  * E = 0 for LW_VARIANT_GENERIC and for f16 at batch 1 and 2 (each weight is decoded exactly and then multiplied:
- * plain fp32 accumulation), for any finite input, and for the batched LW_VARIANT_TILE and LW_VARIANT_MMA on q8_0, q4_0, q5_0, q6_K
- * (exact integer codes times exact activations, block sums scaled in fp32) as long as |x| <= 2^115, which keeps a
- * block's sum of code * x finite.  The streaming variants multiply the integer codes first and apply
+ * plain fp32 accumulation), for any finite input, and for the batched LW_VARIANT_TILE and LW_VARIANT_MMA on
+ * q8_0, q4_0, q5_0 and q6_K (exact integer codes times the activations -- exact in TILE, to 2^-16 of each one's
+ * own magnitude in MMA -- and block sums scaled in fp32) as long as |x| <= 2^115, which keeps a block's sum of
+ * code * x finite.  The streaming variants multiply the integer codes first and apply
  * block scales and offsets to the sums, and LW_VARIANT_IDOT holds the activations as block fixed point
  * (23 bits + sign relative to the largest magnitude in each run of 16 or 32), so an activation that is
  * huge compared with its neighbours and meets a weight that is zero or nearly so leaves an absolute error
  * that S does not cover.  For them
- *     E = c * sum_k What_k * A_k ,   c = 2^-18 (IDOT, the default for the quantised formats; MMA on q4_K / q5_K / q2_K / q4_1 / q5_1), 2^-16 (STREAM),
- *                                    2^-30 (MMA on f16: activations as two f16 terms relative to their block's largest),
+ *     E = c * sum_k What_k * A_k ,   c = 2^-18 (IDOT, the default for the quantised formats; MMA on q4_K, q5_K, q2_K,
+ *                                    q4_1 and q5_1), 2^-16 (STREAM), 2^-30 (MMA on f16: activations as two f16
+ *                                    terms relative to their block's largest),
  * where, over the aligned run of 32 columns that contains k, A_k is the largest |x| and What_k the largest
  * decoded |w|.  This holds for weights made by lw_quantize, and for any block whose scale * code and offset
  * terms are at most four times its largest decoded magnitude.  The constants are worst-case figures (the
@@ -293,6 +295,9 @@ int lw_plan_info(int fmt, int64_t rows, int64_t cols, int* out6);
  * enabled = 2: the same, and the batched tensor-core kernel (LW_VARIANT_MMA) may start streaming W before
  * the previous kernel has completed -- only for weights that no work still pending on the stream writes
  * (model parameters); X and Y are still not touched before.  Other values: LW_ERR_FORMAT.
+ * The batched tensor-core kernel adds into Y, which has to be clear first: with overlap off it is launched
+ * cooperatively (one CTA on every SM) and its CTAs clear Y themselves before a grid-wide barrier; with overlap on a
+ * small clearing kernel is chained in front of it.
  * Default off (0).  Process-wide. */
 int lw_set_overlap(int enabled);
 
