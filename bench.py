@@ -427,9 +427,9 @@ def run_step(args):
     launches_per_step = modes[headline][1]
     mma_possible = batch > 1 and fmt in MMA_FORMATS and all(c % 256 == 0 for _, _, c in shapes)
     if mma_possible and (headline == "grouped" or batch >= 3):
-        # the tensor-core kernel adds into Y: with overlap every mat-vec's Y is cleared by a small kernel of its own in
-        # front (chained by programmatic dependent launch); without, the main kernel clears it itself
-        launches_per_step += 0 if overlap_level == 0 else ncalls
+        # the tensor-core kernel adds into Y: with overlap one small kernel per call clears the call's Y first
+        # (chained by programmatic dependent launch); without, the main kernel clears it itself
+        launches_per_step += 0 if overlap_level == 0 else (len(groups) if headline == "grouped" else ncalls)
 
     # ---- device-resident timing of the headline mode, clocks sampled during it
     for _ in range(max(3, args.warmup)):
