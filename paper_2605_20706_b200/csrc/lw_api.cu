@@ -65,11 +65,11 @@ static bool columnwise(int fmt, int64_t rows, int64_t cols, int batch) {
 
 static int pick_variant(int fmt, int64_t rows, int64_t cols, int batch) {
     const int forced = forced_variant();
-    // batch 2..16: the tensor-core kernel where it applies (every format, cols a multiple of 256, q6_K of 2048, q2_K of 1024;
-    // all columns in one pass over the weights).  Measured on the 8B shapes (ms per step, q4_0, one call per
-    // mat-vec): 2.3 / 2.3 / 2.3 / 3.2 for 3 / 4 / 8 / 16 columns, against 2.2 / 3.7 / 7.3 for 2 / 4 / 8 columns through
-    // the batch-1 kernel and 5.6 / 10.9 for 8 / 16 through the fp32 tile kernel: AUTO takes it from three columns on.  The fp32 tile kernel stays for forced
-    // selection (and for AUTO where only it applies: never, today -- its shapes are a subset).
+    // batch 2..16: the tensor-core kernel where it applies (every format, cols a multiple of 256, q6_K of 2048, q2_K
+    // of 1024; all columns in one pass over the weights).  Measured on the 8B shapes (ms per step, q4_0, one call
+    // per mat-vec): 2.3 / 2.3 / 2.3 / 3.1 for 3 / 4 / 8 / 16 columns, against 2.2 / 3.7 / 7.3 for 2 / 4 / 8 columns
+    // through the batch-1 kernel and 5.6 / 10.9 for 8 / 16 through the fp32 tile kernel: AUTO takes it from three
+    // columns on.  The fp32 tile kernel stays for forced selection.
     if (matvec_mma_supported(fmt, rows, cols, batch) &&
         (forced == LW_VARIANT_MMA || (forced == LW_VARIANT_AUTO && batch >= kMmaMinColumns)))
         return LW_VARIANT_MMA;
