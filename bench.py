@@ -388,11 +388,9 @@ def run_step(args):
         lw.matvec_sequence(fmt_id, seq_arr, seq_ws, stream=stream)
 
     def enqueue_grouped(stream):
-        # batch > 1: one lw_matvec_group_batch call per group (q/k/v together, gate/up together, the rest alone)
-        for g in groups:
-            c = shapes[g[0]][2]
-            lw.matvec_group(fmt_id, c, [(wptr + offs[j], shapes[j][1], xptr + 4 * xoffs[g[0]], yptr + 4 * yoffs[j])
-                                        for j in g], stream, batch=batch)
+        # batch > 1: ONE lw_matvec_sequence_batch call per step, which makes one lw_matvec_group_batch call per group
+        # (q/k/v together, gate/up together, the rest alone)
+        lw.matvec_sequence_batch(fmt_id, seq_arr, batch, stream)
 
     modes = {"launches": (enqueue_launches, len(groups),
                           "one lw_matvec_sequence call per step, run as one grouped launch per phase (q/k/v together, "
@@ -404,8 +402,8 @@ def run_step(args):
              "per-call": (enqueue_per_call, ncalls, "one lw_matvec call per mat-vec (%d launches per step), q/k/v and "
                                                     "gate/up on parallel graph branches" % ncalls),
              "grouped": (enqueue_grouped, len(groups),
-                         "one lw_matvec_group_batch call per group of mat-vecs that share their activations (q/k/v together, "
-                         "gate/up together, the rest alone: %d calls per step)" % len(groups))}
+                         "one lw_matvec_sequence_batch call per step: one launch of the batched kernel per group of mat-vecs that "
+                         "share their activations (q/k/v together, gate/up together, the rest alone: %d per step)" % len(groups))}
     if batch > 1:
         to_time = ["per-call", "grouped"] if args.issue == "auto" else [args.issue]
     elif args.issue == "auto":
@@ -498,15 +496,12 @@ def run_step(args):
         # batch > 1: the caller's two block copies (pinned host memory, same stream) around the step's calls in the
         # headline issue mode -- the C ABI has a host-buffer form of the chain only for batch 1
         def enqueue_block_host(stream):
-            with torch.cuda.stream(stream):
-                X.copy_(X_host, non_blocking=True)
-                modes[headline][0](stream)
-                Y_host.copy_(Y, non_blocking=True)
+            lw.matvec_sequence_batch_host(fmt_id, seq_arr, batch, xhptr, xptr, 4 * xt, yptr, yhptr, 4 * yt, stream)
         ms_host = timer.time(capture(torch, enqueue_block_host, not args.no_graph), args.steps, 3) * args.steps
         h2d, d2h = 4 * xt, 4 * yt
-        e2e_path = "the step's %d-byte activation block from pinned host memory to the device in one copy (issued by the " \
-                   "caller on the same stream), the step's calls (%s), the %d-byte result block back in one copy" % (
-                       4 * xt, headline, 4 * yt)
+        e2e_path = "one lw_matvec_sequence_batch_host call per step: the step's %d-byte activation block from pinned host " \
+                   "memory to the device in one copy, the chain (one grouped call per group), the %d-byte result block " \
+                   "back in one copy" % (4 * xt, 4 * yt)
     lw.set_sequence_mode(lw.SEQ_AUTO)
     if lw.device_status() != 0:
         raise RuntimeError("device fault recorded during the timed region")

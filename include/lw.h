@@ -217,6 +217,19 @@ int lw_matvec_sequence_host(int fmt, int n_items, const lw_seq_item* items, cons
                             int64_t in_bytes, const void* out_dev, void* out_host, int64_t out_bytes, void* workspace,
                             int64_t workspace_bytes, void* stream);
 
+/* The chain with `batch` activation columns per item (1..16): X of an item is batch * cols floats, Y batch * rows,
+ * laid out as in lw_matvec.  Runs of consecutive items that share their X pointer and width and are not flagged
+ * LW_SEQ_DEPENDENT go into one lw_matvec_group_batch call each (one launch of the tensor-core kernel where it
+ * applies); stream order provides every dependency.  No workspace.  Errors as lw_matvec_sequence, LW_ERR_BATCH for
+ * batch outside 1..16; a call that fails validation enqueues nothing. */
+int lw_matvec_sequence_batch(int fmt, int n_items, const lw_seq_item* items, int batch, void* stream);
+
+/* The same with the step's inputs and results in HOST memory, as lw_matvec_sequence_host: in_bytes from in_host to
+ * in_dev first, out_bytes from out_dev to out_host last, all asynchronously on `stream`. */
+int lw_matvec_sequence_batch_host(int fmt, int n_items, const lw_seq_item* items, int batch, const void* in_host,
+                                  void* in_dev, int64_t in_bytes, const void* out_dev, void* out_host, int64_t out_bytes,
+                                  void* stream);
+
 /* Kernel-variant selection [Sec 3.2: the kernel library picks a variant from the tensor context;
  * tunable work-group and tile sizes].  LW_VARIANT_AUTO lets the launch heuristics decide. */
 typedef enum {

@@ -361,6 +361,60 @@ int lw_matvec_sequence_host(int fmt, int n_items, const lw_seq_item* items, cons
     return LW_OK;
 }
 
+static int check_sequence_batch(int fmt, int n_items, const lw_seq_item* items, int batch) {
+    if (lw_block_elems(fmt) == 0) return LW_ERR_FORMAT;
+    if (!items) return LW_ERR_NULL;
+    if (n_items < 1 || n_items > 640) return LW_ERR_SHAPE;
+    for (int j = 0; j < n_items; ++j) {
+        const int rc = check_matvec_args(fmt, items[j].W_blocks, items[j].rows, items[j].cols, items[j].X, items[j].Y, batch);
+        if (rc != LW_OK) return rc;
+        if (items[j].flags & ~LW_SEQ_DEPENDENT) return LW_ERR_FORMAT;
+    }
+    return LW_OK;
+}
+
+int lw_matvec_sequence_batch(int fmt, int n_items, const lw_seq_item* items, int batch, void* stream) {
+    const int rc = check_sequence_batch(fmt, n_items, items, batch);
+    if (rc != LW_OK) return rc;
+    // one grouped call per run of consecutive items that share their X and their width and are not flagged
+    // dependent; stream order provides every dependency
+    int j = 0;
+    while (j < n_items) {
+        int n = 1;
+        while (j + n < n_items && n < 8 && !(items[j + n].flags & LW_SEQ_DEPENDENT) && items[j + n].X == items[j].X &&
+               items[j + n].cols == items[j].cols)
+            ++n;
+        lw_group_item g[8];
+        for (int k = 0; k < n; ++k) {
+            g[k].W_blocks = items[j + k].W_blocks;
+            g[k].rows = items[j + k].rows;
+            g[k].X = items[j + k].X;
+            g[k].Y = items[j + k].Y;
+        }
+        const int rc2 = lw_matvec_group_batch(fmt, items[j].cols, n, g, batch, stream);
+        if (rc2 != LW_OK) return rc2;
+        j += n;
+    }
+    return LW_OK;
+}
+
+int lw_matvec_sequence_batch_host(int fmt, int n_items, const lw_seq_item* items, int batch, const void* in_host,
+                                  void* in_dev, int64_t in_bytes, const void* out_dev, void* out_host, int64_t out_bytes,
+                                  void* stream) {
+    if (!in_host || !in_dev || !out_dev || !out_host) return LW_ERR_NULL;
+    if (in_bytes < 0 || out_bytes < 0) return LW_ERR_SHAPE;
+    const int rc = check_sequence_batch(fmt, n_items, items, batch);      // a call that fails enqueues nothing
+    if (rc != LW_OK) return rc;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (in_bytes > 0 && cudaMemcpyAsync(in_dev, in_host, (size_t)in_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess)
+        return LW_ERR_CUDA;
+    const int rc2 = lw_matvec_sequence_batch(fmt, n_items, items, batch, stream);
+    if (rc2 != LW_OK) return rc2;
+    if (out_bytes > 0 && cudaMemcpyAsync(out_host, out_dev, (size_t)out_bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess)
+        return LW_ERR_CUDA;
+    return LW_OK;
+}
+
 int lw_set_sequence_mode(int mode) {
     if (mode < LW_SEQ_AUTO || mode > LW_SEQ_LAUNCHES) return LW_ERR_FORMAT;
     g_sequence_mode.store(mode);

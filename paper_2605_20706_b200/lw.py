@@ -28,7 +28,7 @@ ERR_WORKSPACE = -9
 LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "liblw.so")
 
 EXPORTS = ("lw_block_elems", "lw_block_bytes", "lw_row_bytes", "lw_status_string", "lw_quantize",
-           "lw_dequant", "lw_matvec", "lw_matvec_group", "lw_matvec_group_batch", "lw_matvec_host", "lw_set_variant", "lw_query_variant",
+           "lw_dequant", "lw_matvec", "lw_matvec_group", "lw_matvec_group_batch", "lw_matvec_sequence_batch", "lw_matvec_sequence_batch_host", "lw_matvec_host", "lw_set_variant", "lw_query_variant",
            "lw_set_overlap", "lw_device_status", "lw_set_tuning", "lw_plan_info", "lw_attn_decode",
            "lw_attn_workspace_bytes", "lw_attn_decode_static", "lw_set_attn_variant", "lw_query_attn_variant",
            "lw_debug_drop_copy", "lw_matvec_sequence", "lw_matvec_sequence_workspace_bytes", "lw_probe_read", "lw_set_sequence_mode", "lw_matvec_sequence_host", "lw_set_shape_tuning", "lw_clear_shape_tuning")
@@ -84,6 +84,10 @@ def lib() -> ctypes.CDLL:
     L.lw_set_sequence_mode.restype, L.lw_set_sequence_mode.argtypes = c_int, [c_int]
     L.lw_matvec_sequence_host.restype = c_int
     L.lw_matvec_sequence_host.argtypes = [c_int, c_int, vp, vp, vp, i64, vp, vp, i64, vp, i64, vp]
+    L.lw_matvec_sequence_batch.restype = c_int
+    L.lw_matvec_sequence_batch.argtypes = [c_int, c_int, vp, c_int, vp]
+    L.lw_matvec_sequence_batch_host.restype = c_int
+    L.lw_matvec_sequence_batch_host.argtypes = [c_int, c_int, vp, c_int, vp, vp, i64, vp, vp, i64, vp]
     L.lw_probe_read.restype, L.lw_probe_read.argtypes = c_int, [vp, i64, vp]
     L.lw_debug_drop_copy.restype, L.lw_debug_drop_copy.argtypes = c_int, [c_int]
     L.lw_attn_decode_static.restype = c_int
@@ -219,6 +223,22 @@ def matvec_sequence_host(fmt: int, items, in_host, in_dev, in_bytes: int, out_de
     _check(lib().lw_matvec_sequence_host(fmt, len(arr), ctypes.cast(arr, ctypes.c_void_p), _addr(in_host), _addr(in_dev),
                                          in_bytes, _addr(out_dev), _addr(out_host), out_bytes, _addr(workspace),
                                          workspace_bytes, _stream_handle(stream)), "lw_matvec_sequence_host")
+
+
+def matvec_sequence_batch(fmt: int, items, batch: int, stream=None) -> None:
+    """A chain of mat-vecs with `batch` columns each: (W_blocks, rows, cols, X, Y, flags) tuples or seq_items()."""
+    arr = items if isinstance(items, ctypes.Array) else seq_items(items)
+    _check(lib().lw_matvec_sequence_batch(fmt, len(arr), ctypes.cast(arr, ctypes.c_void_p), batch, _stream_handle(stream)),
+           "lw_matvec_sequence_batch")
+
+
+def matvec_sequence_batch_host(fmt: int, items, batch: int, in_host, in_dev, in_bytes: int, out_dev, out_host,
+                               out_bytes: int, stream=None) -> None:
+    """matvec_sequence_batch between one copy of the input block host -> device and one of the output block back."""
+    arr = items if isinstance(items, ctypes.Array) else seq_items(items)
+    _check(lib().lw_matvec_sequence_batch_host(fmt, len(arr), ctypes.cast(arr, ctypes.c_void_p), batch, _addr(in_host),
+                                               _addr(in_dev), in_bytes, _addr(out_dev), _addr(out_host), out_bytes,
+                                               _stream_handle(stream)), "lw_matvec_sequence_batch_host")
 
 
 def matvec_host(fmt: int, W_blocks, rows: int, cols: int, X_host, Y_host, X_dev, Y_dev,

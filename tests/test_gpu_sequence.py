@@ -213,3 +213,60 @@ def test_sequence_argument_errors_enqueue_nothing():
     assert L.lw_matvec_sequence(lw.Q8_0, 1, None, lw._addr(ws), 256, None) == lw.ERR_NULL
     torch.cuda.synchronize()
     assert (y == 5.0).all()
+
+
+@pytest.mark.parametrize("overlap", [0, 2])
+@pytest.mark.parametrize("batch", [1, 4, 11])
+@pytest.mark.parametrize("fmt", [lw.Q4_K, lw.Q8_0, lw.F16, lw.Q6_K, lw.Q2_K])
+def test_batched_chain_and_its_host_buffer_form(fmt, batch, overlap):
+    # lw_matvec_sequence_batch: the chain with several columns per item (one grouped call per run of items that share
+    # their X: the tensor-core kernel from two columns on), and lw_matvec_sequence_batch_host around it: the
+    # input block from pinned host memory in one copy, the result block back in one copy
+    lw.set_overlap(overlap)
+    try:
+        spec = [(300, 2048, 0, DEP), (77, 2048, 0, 0), (513, 2048, 0, 0), (256, 2048, 1, DEP), (129, 4096, 2, DEP),
+                (40, 4096, 2, 0)]                                         # rows, cols, which x, flags
+        xs = [synth.activations(170, i, batch, c) for i, c in ((0, 2048), (1, 2048), (2, 4096))]
+        xoff = [0, batch * 2048, 2 * batch * 2048]
+        in_host = torch.from_numpy(np.concatenate([x.reshape(-1) for x in xs])).pin_memory()
+        in_dev = Guarded(in_host.numel())
+        yoff, total = [], 0
+        for rows, _, _, _ in spec:
+            yoff.append(total)
+            total += (batch * rows + 63) & ~63
+        out_dev = Guarded(total)
+        out_host = torch.full((total,), float("nan"), dtype=torch.float32).pin_memory()
+        items, refs, keep = [], [], []
+        for j, (rows, cols, xi, flags) in enumerate(spec):
+            blocks = quantized_weights(fmt, rows, cols, seed=171 + j, tensor_id=fmt)
+            w = torch.from_numpy(blocks).cuda()
+            keep.append(w)
+            items.append((w, rows, cols, in_dev.t.data_ptr() + 4 * xoff[xi], out_dev.t.data_ptr() + 4 * yoff[j], flags))
+            refs.append(oracle.matvec(fmt, blocks, rows, cols, xs[xi], batch, nthreads=4))
+        for _ in range(2):
+            lw.matvec_sequence_batch_host(fmt, items, batch, in_host, in_dev.t, 4 * in_host.numel(), out_dev.t, out_host,
+                                          4 * total)
+        torch.cuda.synchronize()
+        assert lw.device_status() == 0
+        in_dev.check("device input block")
+        out_dev.check("device output block")
+        for j, (rows, _, _, _) in enumerate(spec):
+            got = out_host.numpy()[yoff[j]:yoff[j] + batch * rows].reshape(batch, rows)
+            check_matvec(got, refs[j][0], refs[j][1], "batched chain item %d" % j)
+        # the device-resident form gives the same results
+        out_dev.t.fill_(float("nan"))
+        lw.matvec_sequence_batch(fmt, items, batch)
+        torch.cuda.synchronize()
+        for j, (rows, _, _, _) in enumerate(spec):
+            got = out_dev.t[yoff[j]:yoff[j] + batch * rows].cpu().numpy().reshape(batch, rows)
+            check_matvec(got, refs[j][0], refs[j][1], "batched chain item %d (device)" % j)
+        L = lw.lib()
+        import ctypes
+        arr = lw.seq_items(items)
+        assert L.lw_matvec_sequence_batch(fmt, len(items), ctypes.cast(arr, ctypes.c_void_p), 17, None) == lw.ERR_BATCH
+        assert L.lw_matvec_sequence_batch(fmt, 0, ctypes.cast(arr, ctypes.c_void_p), 4, None) == lw.ERR_SHAPE
+        assert L.lw_matvec_sequence_batch_host(fmt, len(items), ctypes.cast(arr, ctypes.c_void_p), 4, None,
+                                               in_dev.t.data_ptr(), 16, out_dev.t.data_ptr(), out_host.data_ptr(), 16,
+                                               None) == lw.ERR_NULL
+    finally:
+        lw.set_overlap(0)
