@@ -220,7 +220,9 @@ int lw_matvec_sequence_host(int fmt, int n_items, const lw_seq_item* items, cons
 /* The chain with `batch` activation columns per item (1..16): X of an item is batch * cols floats, Y batch * rows,
  * laid out as in lw_matvec.  Runs of consecutive items that share their X pointer and width and are not flagged
  * LW_SEQ_DEPENDENT go into one lw_matvec_group_batch call each (one launch of the tensor-core kernel where it
- * applies); stream order provides every dependency.  No workspace.  Errors as lw_matvec_sequence, LW_ERR_BATCH for
+ * applies); stream order provides every dependency.  Under lw_set_overlap a launch of that kernel also clears the
+ * outputs of the launch after it where they overlap nothing it reads or writes (checked on the host), which saves the
+ * clearing kernel in between.  No workspace.  Errors as lw_matvec_sequence, LW_ERR_BATCH for
  * batch outside 1..16; a call that fails validation enqueues nothing. */
 int lw_matvec_sequence_batch(int fmt, int n_items, const lw_seq_item* items, int batch, void* stream);
 

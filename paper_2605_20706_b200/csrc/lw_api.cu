@@ -236,7 +236,8 @@ int lw_matvec_group_batch(int fmt, int64_t cols, int n_items, const lw_group_ite
     if ((forced == LW_VARIANT_AUTO || forced == LW_VARIANT_MMA) && matvec_mma_group_supported(fmt, cols, n_items, rows, batch)) {
         const int ov = g_overlap.load();
         const int err = launch_matvec_mma_group(fmt, cols, n_items, W, rows, X, Y, batch, ov,
-                                                ov == 0 && cooperative_launch_ok(), static_cast<cudaStream_t>(stream));
+                                                ov == 0 && cooperative_launch_ok(), static_cast<cudaStream_t>(stream), false, 0,
+                                                nullptr, nullptr);
         return err == 0 ? LW_OK : LW_ERR_CUDA;
     }
     for (int j = 0; j < n_items; ++j) {
@@ -373,26 +374,89 @@ static int check_sequence_batch(int fmt, int n_items, const lw_seq_item* items, 
     return LW_OK;
 }
 
+// Do the byte ranges [a, a + na) and [b, b + nb) overlap?
+static bool ranges_overlap(const void* a, int64_t na, const void* b, int64_t nb) {
+    const uintptr_t a0 = reinterpret_cast<uintptr_t>(a), b0 = reinterpret_cast<uintptr_t>(b);
+    return a0 < b0 + (uintptr_t)nb && b0 < a0 + (uintptr_t)na;
+}
+
 int lw_matvec_sequence_batch(int fmt, int n_items, const lw_seq_item* items, int batch, void* stream) {
     const int rc = check_sequence_batch(fmt, n_items, items, batch);
     if (rc != LW_OK) return rc;
-    // one grouped call per run of consecutive items that share their X and their width and are not flagged
-    // dependent; stream order provides every dependency
-    int j = 0;
-    while (j < n_items) {
+    // One grouped call per run of consecutive items that share their X and their width and are not flagged
+    // dependent; stream order provides every dependency.  Where two consecutive runs both take the tensor-core
+    // kernel under lw_set_overlap, and the outputs of the second overlap nothing the first reads or writes, the
+    // first clears them at its end and the second needs no clearing kernel in front of it.
+    const int forced = forced_variant();
+    const int ov = g_overlap.load();
+    const bool mma_allowed = forced == LW_VARIANT_AUTO || forced == LW_VARIANT_MMA;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    auto run_length = [&](int j) {
         int n = 1;
         while (j + n < n_items && n < 8 && !(items[j + n].flags & LW_SEQ_DEPENDENT) && items[j + n].X == items[j].X &&
                items[j + n].cols == items[j].cols)
             ++n;
-        lw_group_item g[8];
-        for (int k = 0; k < n; ++k) {
-            g[k].W_blocks = items[j + k].W_blocks;
-            g[k].rows = items[j + k].rows;
-            g[k].X = items[j + k].X;
-            g[k].Y = items[j + k].Y;
+        return n;
+    };
+    auto takes_mma = [&](int j, int n) {
+        int64_t rows[8];
+        for (int k = 0; k < n; ++k) rows[k] = items[j + k].rows;
+        return mma_allowed && matvec_mma_group_supported(fmt, items[j].cols, n, rows, batch);
+    };
+    int j = 0;
+    bool pre_cleared = false;
+    while (j < n_items) {
+        const int n = run_length(j);
+        const bool mma = takes_mma(j, n);
+        // can this run clear the next run's outputs?
+        int n_next = 0;
+        float* next_y[8];
+        int64_t next_n[8];
+        if (mma && ov >= 1 && j + n < n_items) {
+            const int jn = j + n, nn = run_length(jn);
+            bool ok = takes_mma(jn, nn);
+            for (int a = 0; a < nn && ok; ++a) {
+                const int64_t ybytes = 4 * (int64_t)batch * items[jn + a].rows;
+                for (int b = 0; b < n && ok; ++b)
+                    ok = !ranges_overlap(items[jn + a].Y, ybytes, items[j + b].X, 4 * (int64_t)batch * items[j + b].cols) &&
+                         !ranges_overlap(items[jn + a].Y, ybytes, items[j + b].Y, 4 * (int64_t)batch * items[j + b].rows) &&
+                         !ranges_overlap(items[jn + a].Y, ybytes, items[j + b].W_blocks,
+                                         (int64_t)items[j + b].rows * (int64_t)lw_row_bytes(fmt, items[j + b].cols));
+            }
+            if (ok) {
+                n_next = nn;
+                for (int a = 0; a < nn; ++a) {
+                    next_y[a] = items[jn + a].Y;
+                    next_n[a] = (int64_t)batch * items[jn + a].rows;
+                }
+            }
         }
-        const int rc2 = lw_matvec_group_batch(fmt, items[j].cols, n, g, batch, stream);
-        if (rc2 != LW_OK) return rc2;
+        if (mma) {
+            const void* W[8];
+            const float* X[8];
+            float* Y[8];
+            int64_t rows[8];
+            for (int k = 0; k < n; ++k) {
+                W[k] = items[j + k].W_blocks;
+                X[k] = items[j + k].X;
+                Y[k] = items[j + k].Y;
+                rows[k] = items[j + k].rows;
+            }
+            const int err = launch_matvec_mma_group(fmt, items[j].cols, n, W, rows, X, Y, batch, ov,
+                                                    ov == 0 && cooperative_launch_ok(), s, pre_cleared, n_next, next_y, next_n);
+            if (err != 0) return LW_ERR_CUDA;
+        } else {
+            lw_group_item g[8];
+            for (int k = 0; k < n; ++k) {
+                g[k].W_blocks = items[j + k].W_blocks;
+                g[k].rows = items[j + k].rows;
+                g[k].X = items[j + k].X;
+                g[k].Y = items[j + k].Y;
+            }
+            const int rc2 = lw_matvec_group_batch(fmt, items[j].cols, n, g, batch, stream);
+            if (rc2 != LW_OK) return rc2;
+        }
+        pre_cleared = n_next > 0;
         j += n;
     }
     return LW_OK;

@@ -55,9 +55,12 @@ int launch_matvec_mma(int fmt, const void* W, int64_t rows, int64_t cols, const 
                       int overlap, bool self_clear, cudaStream_t stream);
 // The same for up to eight matrices of one format and width in one launch (each with its own X and Y).
 bool matvec_mma_group_supported(int fmt, int64_t cols, int n_items, const int64_t* rows, int batch);
+// pre_cleared: the launch before on the stream cleared these outputs; next_*: outputs of the launch after, to be
+// cleared by this one at its end (n_next = 0: none).
 int launch_matvec_mma_group(int fmt, int64_t cols, int n_items, const void* const* W, const int64_t* rows,
                             const float* const* X, float* const* Y, int batch, int overlap, bool self_clear,
-                            cudaStream_t stream);
+                            cudaStream_t stream, bool pre_cleared, int n_next, float* const* next_y,
+                            const int64_t* next_n);
 // Tunables of the streaming kernels (0 = automatic) and the geometry they lead to for a shape.
 void set_stream_tuning(int worker_groups, int stages, int stage_kb);
 // Per-shape tunables (all zero erases the entry); make_plan uses them where the process-wide ones are 0.

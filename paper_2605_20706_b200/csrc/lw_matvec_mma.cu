@@ -113,6 +113,11 @@ struct MmaParams {
     uint32_t x_off, w_off;
     uint32_t sx_off, tab_off;   // block sums of the activations and the warps' scale tables (formats that need them)
     int drop_stage;       // testing aid (separate kernel build): the CTA's stage from which on no copy is requested
+    // Outputs of the NEXT launch on the stream, cleared by this one at its end (a chain call passes them when they
+    // overlap nothing this launch reads or writes): the next launch then needs no clearing kernel in front of it.
+    float* next_y[kMmaMaxItems];
+    int64_t next_n[kMmaMaxItems];     // floats
+    int n_next;
 };
 
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
@@ -1189,6 +1194,14 @@ __global__ void __launch_bounds__(kMmaThreads, kCtasPerSm) matvec_mma_kernel(con
         if (lane == 0) mbar_arrive(&empty[slot]);
     }
     if (cur_rs >= 0) flush();
+    // this CTA's share of the next launch's outputs (complete, like everything else here, when this grid completes)
+    for (int it = 0; it < p.n_next; ++it) {
+        const int64_t quads = p.next_n[it] / 4;
+        const int64_t q0 = quads * blockIdx.x / gridDim.x, q1 = quads * (blockIdx.x + 1) / gridDim.x;
+        float4* y4 = reinterpret_cast<float4*>(p.next_y[it]);
+        for (int64_t i = q0 + tid; i < q1; i += kMmaComputeThreads) y4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (blockIdx.x == 0 && tid < (int)(p.next_n[it] - 4 * quads)) p.next_y[it][4 * quads + tid] = 0.f;
+    }
 }
 
 template <class T, int NT, bool DROP = false>
@@ -1329,11 +1342,15 @@ bool matvec_mma_group_supported(int fmt, int64_t cols, int n_items, const int64_
 // overlap: 0 ordinary launches; 1 programmatic dependent launch (set-up overlaps the previous kernel's end);
 // 2 the same, and the weight copies start before the previous kernel has completed.  self_clear: one cooperative
 // launch whose CTAs clear Y themselves (no clearing kernel, no programmatic launch).
+// pre_cleared: the launch before this one on the stream has cleared these outputs (no clearing of any kind here);
+// n_next / next_y / next_n: outputs of the launch after this one, to be cleared by this one at its end.
 int launch_matvec_mma_group(int fmt, int64_t cols, int n_items, const void* const* W, const int64_t* rows,
                             const float* const* X, float* const* Y, int batch, int overlap, bool self_clear,
-                            cudaStream_t stream) {
+                            cudaStream_t stream, bool pre_cleared, int n_next, float* const* next_y,
+                            const int64_t* next_n) {
     int* fault = device_fault_word();
     if (!fault) return (int)cudaErrorInvalidValue;
+    if (pre_cleared) self_clear = false;
     {
         // The grid barrier of the self-clearing form is one pair of words per device: it relies on two such
         // launches never running at the same time, which holds because each needs every SM to itself (cooperative
@@ -1349,7 +1366,7 @@ int launch_matvec_mma_group(int fmt, int64_t cols, int n_items, const void* cons
     if (self_clear && cudaGetSymbolAddress(reinterpret_cast<void**>(&grid_bar), g_mma_grid_barrier) != cudaSuccess)
         return (int)cudaErrorInvalidValue;
     // the kernel adds every (chunk, row stage) share into Y: clear it first (Y is 16-byte aligned)
-    if (!self_clear) {
+    if (!self_clear && !pre_cleared) {
         ZeroList z{};
         int64_t most = 0;
         for (int i = 0; i < n_items; ++i) {
@@ -1412,6 +1429,11 @@ int launch_matvec_mma_group(int fmt, int64_t cols, int n_items, const void* cons
     int grid = kCtasPerSm * mma_sm_count();
     if ((int64_t)grid > n_stages && !self_clear) grid = (int)n_stages;   // self-clearing: every SM, so launches never overlap
     p.drop_stage = -1;
+    p.n_next = n_next;
+    for (int i = 0; i < n_next; ++i) {
+        p.next_y[i] = next_y[i];
+        p.next_n[i] = next_n[i];
+    }
     if (fmt == LW_Q4_0 && nt == 1) {
         // testing aid: a pending lw_debug_drop_copy request is consumed by this launch
         const int drop = take_drop_unit();
@@ -1453,7 +1475,8 @@ int launch_matvec_mma_group(int fmt, int64_t cols, int n_items, const void* cons
 
 int launch_matvec_mma(int fmt, const void* W, int64_t rows, int64_t cols, const float* X, float* Y, int batch,
                       int overlap, bool self_clear, cudaStream_t stream) {
-    return launch_matvec_mma_group(fmt, cols, 1, &W, &rows, &X, &Y, batch, overlap, self_clear, stream);
+    return launch_matvec_mma_group(fmt, cols, 1, &W, &rows, &X, &Y, batch, overlap, self_clear, stream, false, 0, nullptr,
+                                   nullptr);
 }
 
 }  // namespace lw

@@ -270,3 +270,36 @@ def test_batched_chain_and_its_host_buffer_form(fmt, batch, overlap):
                                                None) == lw.ERR_NULL
     finally:
         lw.set_overlap(0)
+
+
+@pytest.mark.parametrize("overlap", [0, 2])
+def test_batched_chain_over_ping_pong_buffers(overlap):
+    # every item's Y is the buffer the item before it read its X from: the chain call must not let a launch clear
+    # the next launch's outputs here (they overlap its own input) and falls back to the clearing kernel
+    fmt, batch, dims = lw.Q4_0, 6, [1024, 768, 2048, 512, 1024]
+    mats = [quantized_weights(fmt, dims[j + 1], dims[j], seed=180 + j, tensor_id=fmt) for j in range(len(dims) - 1)]
+    wd = [torch.from_numpy(m).cuda() for m in mats]
+    x0 = synth.activations(180, 0, batch, dims[0])
+    bufs = [Guarded(batch * max(dims)), Guarded(batch * max(dims))]
+    bufs[0].t[:x0.size] = torch.from_numpy(x0.reshape(-1)).cuda()
+    items = [(wd[j], dims[j + 1], dims[j], bufs[j & 1].t, bufs[(j + 1) & 1].t, DEP) for j in range(len(mats))]
+    lw.set_overlap(overlap)
+    try:
+        lw.matvec_sequence_batch(fmt, items, batch)
+        torch.cuda.synchronize()
+        assert lw.device_status() == 0
+        for b in bufs:
+            b.check("ping-pong buffer")
+        # the last layer against the oracle fed with the GPU's own input to that layer
+        x_in = bufs[(len(mats) - 1) & 1].t[:batch * dims[-2]].cpu().numpy().reshape(batch, dims[-2])
+        got = bufs[len(mats) & 1].t[:batch * dims[-1]].cpu().numpy().reshape(batch, dims[-1])
+        y_ref, s_ref = oracle.matvec(fmt, mats[-1], dims[-1], dims[-2], x_in, batch, nthreads=4)
+        check_matvec(got, y_ref, s_ref, "ping-pong chain")
+        # and the first layer, recomputed alone
+        y1 = Guarded((batch, dims[1]))
+        lw.matvec(fmt, wd[0], dims[1], dims[0], torch.from_numpy(x0).cuda(), y1.t, batch)
+        torch.cuda.synchronize()
+        y_ref, s_ref = oracle.matvec(fmt, mats[0], dims[1], dims[0], x0, batch, nthreads=4)
+        check_matvec(y1.t.cpu().numpy(), y_ref, s_ref, "first layer")
+    finally:
+        lw.set_overlap(0)
