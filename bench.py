@@ -474,7 +474,7 @@ def run_step(args):
 
     # ---- end to end through the host-buffer entry points of the C ABI, pinned host memory on both sides, the
     # copies inside the timed region.  Batch 1: ONE lw_matvec_sequence_host call per step (the step's activation
-    # block in with one copy, the chain in the headline mode, the result block out with one copy).  Beside it
+    # block in, the chain in the headline mode, the result block out; copies in pieces beside the kernels).  Beside it
     # (and alone for batch > 1): one lw_matvec_host call per mat-vec, each with its own two copies.
     def enqueue_host(stream):
         for i, (_, r, c) in enumerate(shapes):
@@ -490,18 +490,20 @@ def run_step(args):
         ms_host = timer.time(capture(torch, enqueue_seq_host, not args.no_graph), args.steps, 3) * args.steps
         h2d, d2h = 4 * xt, 4 * yt
         e2e_path = "one lw_matvec_sequence_host call per step: the step's %d-byte activation block from pinned host " \
-                   "memory to the device in one copy, the chain (%s), the %d-byte result block back in one copy" % (
+                   "memory to the device, the chain (%s), the %d-byte result block back to pinned host memory; the " \
+                   "library moves both blocks in pieces on its own copy streams beside the kernels (a launch waits " \
+                   "for the pieces it reads; a piece of results leaves when no later mat-vec writes into it)" % (
                        4 * xt, headline, 4 * yt)
     else:
-        # batch > 1: the caller's two block copies (pinned host memory, same stream) around the step's calls in the
-        # headline issue mode -- the C ABI has a host-buffer form of the chain only for batch 1
+        # batch > 1: the host-buffer form of the batched chain
         def enqueue_block_host(stream):
             lw.matvec_sequence_batch_host(fmt_id, seq_arr, batch, xhptr, xptr, 4 * xt, yptr, yhptr, 4 * yt, stream)
         ms_host = timer.time(capture(torch, enqueue_block_host, not args.no_graph), args.steps, 3) * args.steps
         h2d, d2h = 4 * xt, 4 * yt
         e2e_path = "one lw_matvec_sequence_batch_host call per step: the step's %d-byte activation block from pinned host " \
-                   "memory to the device in one copy, the chain (one grouped call per group), the %d-byte result block " \
-                   "back in one copy" % (4 * xt, 4 * yt)
+                   "memory to the device, the chain (one grouped call per group), the %d-byte result block back to " \
+                   "pinned host memory; the library moves both blocks in pieces on its own copy streams beside the " \
+                   "kernels" % (4 * xt, 4 * yt)
     lw.set_sequence_mode(lw.SEQ_AUTO)
     if lw.device_status() != 0:
         raise RuntimeError("device fault recorded during the timed region")

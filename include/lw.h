@@ -207,11 +207,21 @@ typedef enum { LW_SEQ_AUTO = 0, LW_SEQ_PERSISTENT = 1, LW_SEQ_LAUNCHES = 2 } lw_
 /* Process-wide choice of the implementation behind lw_matvec_sequence; LW_ERR_FORMAT for another value. */
 int lw_set_sequence_mode(int mode);
 
-/* lw_matvec_sequence with HOST activations and results: copies in_bytes from in_host to in_dev (one copy: the
- * block that holds the chain's input activations; the items' X pointers point into in_dev), runs the chain,
- * copies out_bytes from out_dev to out_host (the block the items' Y pointers point into), all asynchronously
- * on `stream` (pinned host memory makes the copies truly asynchronous).  in_dev / out_dev are caller-provided
- * device buffers; a size of 0 skips that copy.  The caller synchronises the stream before reading out_host.
+/* lw_matvec_sequence with HOST activations and results: copies in_bytes from in_host to in_dev (the block that
+ * holds the chain's input activations; the items' X pointers point into in_dev), runs the chain, copies out_bytes
+ * from out_dev to out_host (the block the items' Y pointers point into).  In stream order the call is one
+ * operation on `stream`: it starts after everything enqueued before it and `stream` has finished it when both
+ * blocks are complete; it is asynchronous (pinned host memory makes the copies truly asynchronous) and can be
+ * captured into a CUDA graph.  The result is that of one copy in, the chain, one copy out.  Blocks above 128 KB
+ * move in pieces on two copy streams of the library beside the kernels (LW_SEQ_LAUNCHES only): the input block in
+ * address order, a launch waiting only for the pieces up to the end of the activations it reads; a piece of the
+ * result block as soon as no later item writes into it.  Activations and results laid out in the order of the
+ * items overlap best; any layout is correct.  When an item writes into the input block, that block is copied
+ * whole before the first kernel.  in_host must not change and out_host must not be read until the stream has
+ * finished the call.  in_dev / out_dev are caller-provided device buffers; a size of 0 skips that copy.
+ * The library creates its copy streams and events at the first call that needs them (per device) and keeps them;
+ * concurrent calls from several host threads are safe, but while a stream that runs such a call is being
+ * captured no other thread may issue one.
  * Errors as lw_matvec_sequence; a call that fails validation enqueues nothing. */
 int lw_matvec_sequence_host(int fmt, int n_items, const lw_seq_item* items, const void* in_host, void* in_dev,
                             int64_t in_bytes, const void* out_dev, void* out_host, int64_t out_bytes, void* workspace,
@@ -226,8 +236,8 @@ int lw_matvec_sequence_host(int fmt, int n_items, const lw_seq_item* items, cons
  * batch outside 1..16; a call that fails validation enqueues nothing. */
 int lw_matvec_sequence_batch(int fmt, int n_items, const lw_seq_item* items, int batch, void* stream);
 
-/* The same with the step's inputs and results in HOST memory, as lw_matvec_sequence_host: in_bytes from in_host to
- * in_dev first, out_bytes from out_dev to out_host last, all asynchronously on `stream`. */
+/* The same with the step's inputs and results in HOST memory, as lw_matvec_sequence_host (blocks above 128 KB move
+ * in pieces beside the kernels; same rules). */
 int lw_matvec_sequence_batch_host(int fmt, int n_items, const lw_seq_item* items, int batch, const void* in_host,
                                   void* in_dev, int64_t in_bytes, const void* out_dev, void* out_host, int64_t out_bytes,
                                   void* stream);

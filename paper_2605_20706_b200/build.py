@@ -14,7 +14,7 @@ CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(ROOT, "include")
 LIB = os.path.join(HERE, "liblw.so")
 
-SOURCES = ["lw_matvec_stream.cu", "lw_matvec_seq.cu", "lw_matvec_tile.cu", "lw_matvec_mma.cu", "lw_probe.cu", "lw_attn.cu", "lw_api.cu", "lw_dequant.cu", "lw_matvec_generic.cu", "lw_quantize.cpp"]
+SOURCES = ["lw_matvec_stream.cu", "lw_matvec_seq.cu", "lw_matvec_tile.cu", "lw_matvec_mma.cu", "lw_probe.cu", "lw_attn.cu", "lw_api.cu", "lw_hostpipe.cu", "lw_dequant.cu", "lw_matvec_generic.cu", "lw_quantize.cpp"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC"]
 

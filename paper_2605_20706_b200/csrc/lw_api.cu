@@ -283,8 +283,7 @@ int lw_matvec_group(int fmt, int64_t cols, int n_items, const lw_group_item* ite
 
 int64_t lw_matvec_sequence_workspace_bytes(void) { return 256; }
 
-int lw_matvec_sequence(int fmt, int n_items, const lw_seq_item* items, void* workspace, int64_t workspace_bytes,
-                       void* stream) {
+static int check_sequence(int fmt, int n_items, const lw_seq_item* items, void* workspace, int64_t workspace_bytes) {
     if (lw_block_elems(fmt) == 0) return LW_ERR_FORMAT;
     if (!items || !workspace) return LW_ERR_NULL;
     if (n_items < 1 || n_items > 640) return LW_ERR_SHAPE;
@@ -295,13 +294,24 @@ int lw_matvec_sequence(int fmt, int n_items, const lw_seq_item* items, void* wor
         if (rc != LW_OK) return rc;
         if (items[j].flags & ~LW_SEQ_DEPENDENT) return LW_ERR_FORMAT;
     }
+    return LW_OK;
+}
+
+// The chain, arguments already checked.  `pipe` (may be null) carries the copies of the host form: it is told
+// before and behind every launch which items the launch runs.
+static int run_sequence(int fmt, int n_items, const lw_seq_item* items, void* workspace, void* stream, HostPipe* pipe) {
     const bool can = cooperative_launch_ok();
     const bool streaming = forced_variant() == LW_VARIANT_AUTO && matvec_sequence_supported(fmt, n_items, items);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (streaming && can && g_sequence_mode.load() == LW_SEQ_PERSISTENT) {
+        // one kernel for the whole chain: nothing to overlap copies with from the host
+        if (pipe) pipe->whole_copies_only();
+        if (pipe && !pipe->begin()) return LW_ERR_CUDA;
         const int err = launch_matvec_sequence(fmt, n_items, items, static_cast<unsigned*>(workspace), s);
-        return err == 0 ? LW_OK : LW_ERR_CUDA;
+        if (err != 0) return LW_ERR_CUDA;
+        return !pipe || pipe->end() ? LW_OK : LW_ERR_CUDA;
     }
+    if (pipe && !pipe->begin()) return LW_ERR_CUDA;
     if (streaming) {
         // One launch per phase (consecutive items that share their X and are not flagged dependent), chained
         // with programmatic dependent launch: stream order provides every dependency, and a kernel waits for
@@ -322,18 +332,28 @@ int lw_matvec_sequence(int fmt, int n_items, const lw_seq_item* items, void* wor
                 Y[k] = items[j + k].Y;
                 rows[k] = items[j + k].rows;
             }
+            if (pipe && !pipe->before(j, n)) return LW_ERR_CUDA;
             const int err = n == 1 ? launch_matvec_stream(fmt, fmt != LW_F16, W[0], rows[0], items[j].cols, X[0], Y[0], true, s)
                                    : launch_matvec_stream_group(fmt, fmt != LW_F16, items[j].cols, n, W, rows, X, Y, true, s);
             if (err != 0) return LW_ERR_CUDA;
+            if (pipe && !pipe->after(j, n)) return LW_ERR_CUDA;
             j += n;
         }
-        return LW_OK;
+        return !pipe || pipe->end() ? LW_OK : LW_ERR_CUDA;
     }
     for (int j = 0; j < n_items; ++j) {
+        if (pipe && !pipe->before(j, 1)) return LW_ERR_CUDA;
         const int rc = lw_matvec(fmt, items[j].W_blocks, items[j].rows, items[j].cols, items[j].X, items[j].Y, 1, stream);
         if (rc != LW_OK) return rc;
+        if (pipe && !pipe->after(j, 1)) return LW_ERR_CUDA;
     }
-    return LW_OK;
+    return !pipe || pipe->end() ? LW_OK : LW_ERR_CUDA;
+}
+
+int lw_matvec_sequence(int fmt, int n_items, const lw_seq_item* items, void* workspace, int64_t workspace_bytes,
+                       void* stream) {
+    const int rc = check_sequence(fmt, n_items, items, workspace, workspace_bytes);
+    return rc != LW_OK ? rc : run_sequence(fmt, n_items, items, workspace, stream, nullptr);
 }
 
 int lw_matvec_sequence_host(int fmt, int n_items, const lw_seq_item* items, const void* in_host, void* in_dev,
@@ -342,24 +362,10 @@ int lw_matvec_sequence_host(int fmt, int n_items, const lw_seq_item* items, cons
     if (!in_host || !in_dev || !out_dev || !out_host) return LW_ERR_NULL;
     if (in_bytes < 0 || out_bytes < 0) return LW_ERR_SHAPE;
     // validate everything before the first copy is queued: a call that fails enqueues nothing
-    if (lw_block_elems(fmt) == 0) return LW_ERR_FORMAT;
-    if (!items || !workspace) return LW_ERR_NULL;
-    if (n_items < 1 || n_items > 640) return LW_ERR_SHAPE;
-    if (misaligned16(workspace)) return LW_ERR_ALIGN;
-    if (workspace_bytes < lw_matvec_sequence_workspace_bytes()) return LW_ERR_WORKSPACE;
-    for (int j = 0; j < n_items; ++j) {
-        const int rc = check_matvec_args(fmt, items[j].W_blocks, items[j].rows, items[j].cols, items[j].X, items[j].Y, 1);
-        if (rc != LW_OK) return rc;
-        if (items[j].flags & ~LW_SEQ_DEPENDENT) return LW_ERR_FORMAT;
-    }
-    cudaStream_t s = static_cast<cudaStream_t>(stream);
-    if (in_bytes > 0 && cudaMemcpyAsync(in_dev, in_host, (size_t)in_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess)
-        return LW_ERR_CUDA;
-    const int rc = lw_matvec_sequence(fmt, n_items, items, workspace, workspace_bytes, stream);
+    const int rc = check_sequence(fmt, n_items, items, workspace, workspace_bytes);
     if (rc != LW_OK) return rc;
-    if (out_bytes > 0 && cudaMemcpyAsync(out_host, out_dev, (size_t)out_bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess)
-        return LW_ERR_CUDA;
-    return LW_OK;
+    HostPipe pipe(n_items, items, 1, in_host, in_dev, in_bytes, out_dev, out_host, out_bytes, static_cast<cudaStream_t>(stream));
+    return run_sequence(fmt, n_items, items, workspace, stream, &pipe);
 }
 
 static int check_sequence_batch(int fmt, int n_items, const lw_seq_item* items, int batch) {
@@ -380,9 +386,7 @@ static bool ranges_overlap(const void* a, int64_t na, const void* b, int64_t nb)
     return a0 < b0 + (uintptr_t)nb && b0 < a0 + (uintptr_t)na;
 }
 
-int lw_matvec_sequence_batch(int fmt, int n_items, const lw_seq_item* items, int batch, void* stream) {
-    const int rc = check_sequence_batch(fmt, n_items, items, batch);
-    if (rc != LW_OK) return rc;
+static int run_sequence_batch(int fmt, int n_items, const lw_seq_item* items, int batch, void* stream, HostPipe* pipe) {
     // One grouped call per run of consecutive items that share their X and their width and are not flagged
     // dependent; stream order provides every dependency.  Where two consecutive runs both take the tensor-core
     // kernel under lw_set_overlap, and the outputs of the second overlap nothing the first reads or writes, the
@@ -405,9 +409,11 @@ int lw_matvec_sequence_batch(int fmt, int n_items, const lw_seq_item* items, int
     };
     int j = 0;
     bool pre_cleared = false;
+    if (pipe && !pipe->begin()) return LW_ERR_CUDA;
     while (j < n_items) {
         const int n = run_length(j);
         const bool mma = takes_mma(j, n);
+        if (pipe && !pipe->before(j, n)) return LW_ERR_CUDA;
         // can this run clear the next run's outputs?
         int n_next = 0;
         float* next_y[8];
@@ -456,10 +462,16 @@ int lw_matvec_sequence_batch(int fmt, int n_items, const lw_seq_item* items, int
             const int rc2 = lw_matvec_group_batch(fmt, items[j].cols, n, g, batch, stream);
             if (rc2 != LW_OK) return rc2;
         }
+        if (pipe && !pipe->after(j, n)) return LW_ERR_CUDA;
         pre_cleared = n_next > 0;
         j += n;
     }
-    return LW_OK;
+    return !pipe || pipe->end() ? LW_OK : LW_ERR_CUDA;
+}
+
+int lw_matvec_sequence_batch(int fmt, int n_items, const lw_seq_item* items, int batch, void* stream) {
+    const int rc = check_sequence_batch(fmt, n_items, items, batch);
+    return rc != LW_OK ? rc : run_sequence_batch(fmt, n_items, items, batch, stream, nullptr);
 }
 
 int lw_matvec_sequence_batch_host(int fmt, int n_items, const lw_seq_item* items, int batch, const void* in_host,
@@ -469,14 +481,8 @@ int lw_matvec_sequence_batch_host(int fmt, int n_items, const lw_seq_item* items
     if (in_bytes < 0 || out_bytes < 0) return LW_ERR_SHAPE;
     const int rc = check_sequence_batch(fmt, n_items, items, batch);      // a call that fails enqueues nothing
     if (rc != LW_OK) return rc;
-    cudaStream_t s = static_cast<cudaStream_t>(stream);
-    if (in_bytes > 0 && cudaMemcpyAsync(in_dev, in_host, (size_t)in_bytes, cudaMemcpyHostToDevice, s) != cudaSuccess)
-        return LW_ERR_CUDA;
-    const int rc2 = lw_matvec_sequence_batch(fmt, n_items, items, batch, stream);
-    if (rc2 != LW_OK) return rc2;
-    if (out_bytes > 0 && cudaMemcpyAsync(out_host, out_dev, (size_t)out_bytes, cudaMemcpyDeviceToHost, s) != cudaSuccess)
-        return LW_ERR_CUDA;
-    return LW_OK;
+    HostPipe pipe(n_items, items, batch, in_host, in_dev, in_bytes, out_dev, out_host, out_bytes, static_cast<cudaStream_t>(stream));
+    return run_sequence_batch(fmt, n_items, items, batch, stream, &pipe);
 }
 
 int lw_set_sequence_mode(int mode) {

@@ -84,6 +84,36 @@ void set_attn_variant(int variant);
 int attn_variant_of(int fmt, int64_t n_head, int64_t n_kv_head, int64_t head_dim, int64_t n_pos);
 // Address of the per-device fault word (device memory), or nullptr on error.
 int* device_fault_word();
+
+// Host <-> device copies of a chain's input and result blocks, in pieces that overlap with the chain's kernels
+// (lw_hostpipe.cu).  The chain code calls begin() first, before(j, n) ahead of the launch that runs items
+// j .. j+n-1, after(j, n) behind it, and end() last; every call returns false on a CUDA error.
+class HostPipe {
+public:
+    HostPipe(int n_items, const lw_seq_item* items, int batch, const void* in_host, void* in_dev, int64_t in_bytes,
+             const void* out_dev, void* out_host, int64_t out_bytes, cudaStream_t stream);
+    ~HostPipe();
+    HostPipe(const HostPipe&) = delete;
+    HostPipe& operator=(const HostPipe&) = delete;
+    void whole_copies_only();      // one copy in before the first kernel, one copy out behind the last (call before begin)
+    bool begin();
+    bool before(int j, int n);     // the caller's stream waits for the input pieces these items read
+    bool after(int j, int n);      // result pieces that no later item writes may leave
+    bool end();                    // the rest of both blocks; the caller's stream waits for all copies
+private:
+    struct State;
+    cudaEvent_t event();
+    bool copy_in(int64_t upto);
+    bool copy_out(int64_t upto);
+    const char* in_host_;
+    char* in_dev_;
+    int64_t in_bytes_;
+    const char* out_dev_;
+    char* out_host_;
+    int64_t out_bytes_;
+    cudaStream_t s_;
+    State* st_;
+};
 #endif
 
 }  // namespace lw

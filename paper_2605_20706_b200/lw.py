@@ -216,7 +216,8 @@ def set_sequence_mode(mode: int) -> None:
 
 def matvec_sequence_host(fmt: int, items, in_host, in_dev, in_bytes: int, out_dev, out_host, out_bytes: int, workspace,
                          workspace_bytes: int | None = None, stream=None) -> None:
-    """matvec_sequence between one copy of the input block host -> device and one of the output block back."""
+    """matvec_sequence with the input block in host memory and the result block returned to host memory (the
+    library overlaps the copies with the kernels)."""
     arr = items if isinstance(items, ctypes.Array) else seq_items(items)
     if workspace_bytes is None:
         workspace_bytes = workspace.numel() * workspace.element_size() if hasattr(workspace, "numel") else 0
@@ -234,7 +235,7 @@ def matvec_sequence_batch(fmt: int, items, batch: int, stream=None) -> None:
 
 def matvec_sequence_batch_host(fmt: int, items, batch: int, in_host, in_dev, in_bytes: int, out_dev, out_host,
                                out_bytes: int, stream=None) -> None:
-    """matvec_sequence_batch between one copy of the input block host -> device and one of the output block back."""
+    """matvec_sequence_batch with the input block in host memory and the result block returned to host memory."""
     arr = items if isinstance(items, ctypes.Array) else seq_items(items)
     _check(lib().lw_matvec_sequence_batch_host(fmt, len(arr), ctypes.cast(arr, ctypes.c_void_p), batch, _addr(in_host),
                                                _addr(in_dev), in_bytes, _addr(out_dev), _addr(out_host), out_bytes,

@@ -303,3 +303,113 @@ def test_batched_chain_over_ping_pong_buffers(overlap):
         check_matvec(y1.t.cpu().numpy(), y_ref, s_ref, "first layer")
     finally:
         lw.set_overlap(0)
+
+
+def _host_chain(fmt, batch, layout, n_items=24, rows=1500, cols=4096, seed=190):
+    """A chain of dependent items with one X each, the X in the input block and the Y in the result block in the
+    order `layout` gives; with "hole", item 0 writes into a gap of the input block instead."""
+    order = list(range(n_items))
+    if layout == "descending":
+        order = order[::-1]
+    elif layout == "shuffled":
+        order = [int(v) for v in np.random.default_rng(5).permutation(n_items)]
+    xw, yw = batch * cols, (batch * rows + 63) & ~63
+    hole = yw if layout == "hole" else 0
+    in_words, out_words = n_items * xw + hole, n_items * yw
+    in_np = np.full(in_words, np.nan, dtype=np.float32)
+    xs, items, refs, keep = [], [], [], []
+    in_dev, out_dev = Guarded(in_words), Guarded(out_words)
+    for j in range(n_items):
+        X = synth.activations(seed, j, batch, cols)
+        in_np[order[j] * xw:(order[j] + 1) * xw] = X.reshape(-1)
+        blocks = quantized_weights(fmt, rows, cols, seed=seed + 1 + j, tensor_id=fmt)
+        w = torch.from_numpy(blocks).cuda()
+        keep.append(w)
+        y_ptr = out_dev.t.data_ptr() + 4 * order[j] * yw
+        if hole and j == 0:
+            y_ptr = in_dev.t.data_ptr() + 4 * n_items * xw         # behind every X: the last piece of a piecewise copy
+        items.append((w, rows, cols, in_dev.t.data_ptr() + 4 * order[j] * xw, y_ptr, DEP))
+        refs.append(oracle.matvec(fmt, blocks, rows, cols, X, batch, nthreads=4))
+    in_host = torch.from_numpy(in_np).pin_memory()
+    out_host = torch.full((out_words,), float("nan"), dtype=torch.float32).pin_memory()
+    return dict(items=items, refs=refs, keep=keep, in_host=in_host, in_dev=in_dev, out_dev=out_dev, out_host=out_host,
+                order=order, yw=yw, xw=xw, rows=rows, hole=hole, n=n_items, batch=batch)
+
+
+def _check_host_chain(c, what):
+    torch.cuda.synchronize()
+    assert lw.device_status() == 0
+    c["in_dev"].check("device input block")
+    c["out_dev"].check("device output block")
+    batch, rows = c["batch"], c["rows"]
+    for j in range(c["n"]):
+        if c["hole"] and j == 0:
+            got = c["in_dev"].t[c["n"] * c["xw"]:c["n"] * c["xw"] + batch * rows].cpu().numpy()
+        else:
+            got = c["out_host"].numpy()[c["order"][j] * c["yw"]:c["order"][j] * c["yw"] + batch * rows]
+        check_matvec(got.reshape(batch, rows), c["refs"][j][0], c["refs"][j][1], "%s item %d" % (what, j))
+    # the whole input block is on the device afterwards, whether an item read it or not
+    n_x = c["n"] * c["xw"]
+    assert torch.equal(c["in_dev"].t[:n_x].cpu(), c["in_host"][:n_x])
+
+
+@pytest.mark.parametrize("graph", [False, True])
+@pytest.mark.parametrize("layout", ["ascending", "descending", "shuffled", "hole"])
+@pytest.mark.parametrize("mode", MODES)
+def test_host_chain_whose_blocks_are_copied_in_pieces(mode, layout, graph):
+    # blocks of several hundred KB: the input block goes in piece by piece beside the kernels and the result block
+    # leaves piece by piece; whatever the order of the activations and results inside the blocks, the outcome is
+    # that of one copy before and one copy behind the chain.  "hole": an item writes into the input block, which
+    # a late piece must not overwrite.
+    lw.set_sequence_mode(mode)
+    fmt = lw.Q4_K
+    c = _host_chain(fmt, 1, layout)
+    ws = _workspace()
+
+    def call(stream=None):
+        lw.matvec_sequence_host(fmt, c["items"], c["in_host"], c["in_dev"].t, 4 * c["in_host"].numel(), c["out_dev"].t,
+                                c["out_host"], 4 * c["out_host"].numel(), ws.t, stream=stream)
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        call(side)
+        side.synchronize()
+        _check_host_chain(c, "eager")
+        if graph:
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=side):
+                call(side)
+            for _ in range(3):
+                c["out_host"].fill_(float("nan"))
+                c["in_dev"].t.fill_(float("nan"))
+                g.replay()
+                torch.cuda.synchronize()
+                _check_host_chain(c, "replay")
+
+
+@pytest.mark.parametrize("overlap", [0, 2])
+@pytest.mark.parametrize("layout", ["ascending", "shuffled", "hole"])
+@pytest.mark.parametrize("fmt,batch", [(lw.Q4_0, 3), (lw.Q8_0, 8), (lw.F16, 2)])
+def test_batched_host_chain_whose_blocks_are_copied_in_pieces(fmt, batch, layout, overlap):
+    lw.set_overlap(overlap)
+    try:
+        c = _host_chain(fmt, batch, layout, n_items=12, rows=700, cols=2048, seed=230)
+        side = torch.cuda.Stream()
+
+        def call(stream):
+            lw.matvec_sequence_batch_host(fmt, c["items"], batch, c["in_host"], c["in_dev"].t, 4 * c["in_host"].numel(),
+                                          c["out_dev"].t, c["out_host"], 4 * c["out_host"].numel(), stream)
+        with torch.cuda.stream(side):
+            call(side)
+            side.synchronize()
+            _check_host_chain(c, "eager")
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=side):
+                call(side)
+            for _ in range(2):
+                c["out_host"].fill_(float("nan"))
+                c["in_dev"].t.fill_(float("nan"))
+                g.replay()
+                torch.cuda.synchronize()
+                _check_host_chain(c, "replay")
+    finally:
+        lw.set_overlap(0)
