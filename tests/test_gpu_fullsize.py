@@ -87,3 +87,55 @@ def test_llama8b_gate_batched(batch):
     idx = _sample_rows(rows, np.random.default_rng(batch), n=400)
     y_ref, s_ref = oracle.matvec(fmt, blocks, rows, cols, X, batch, nthreads=8, row_idx=idx)
     check_matvec(y.cpu().numpy()[:, idx], y_ref, s_ref, "batched gate, batch %d" % batch)
+
+
+LAYER_8B = [("q", 4096, 4096, 0), ("k", 1024, 4096, 0), ("v", 1024, 4096, 0), ("o", 4096, 4096, 1),
+            ("gate", 14336, 4096, 2), ("up", 14336, 4096, 2), ("down", 4096, 14336, 3), ("lm_head", 128256, 4096, 4)]
+LAYER_1B = [("q", 2048, 2048, 0), ("k", 512, 2048, 0), ("v", 512, 2048, 0), ("o", 2048, 2048, 1),
+            ("gate", 8192, 2048, 2), ("up", 8192, 2048, 2), ("down", 2048, 8192, 3), ("lm_head", 128256, 2048, 4)]
+
+
+@pytest.mark.parametrize("fmt,batch,layer", [(lw.Q4_0, 8, LAYER_8B), (lw.Q4_0, 16, LAYER_8B), (lw.Q8_0, 16, LAYER_8B),
+                                             (lw.Q4_K, 8, LAYER_8B), (lw.Q6_K, 16, LAYER_8B), (lw.Q2_K, 5, LAYER_8B),
+                                             (lw.F16, 8, LAYER_1B), (lw.F16, 16, LAYER_1B)])
+def test_layer_and_lm_head_batched_chain(fmt, batch, layer):
+    # the batched step as bench.py issues it: one lw_matvec_sequence_batch call over a layer's mat-vecs and lm_head
+    # at their full sizes (q/k/v and gate/up share their activations), weights requested ahead of the dependency
+    # wait (overlap level 2), replayed as a CUDA graph; sampled rows of every matrix against the oracle
+    xs, items, keep, cases = {}, [], [], []
+    for j, (name, rows, cols, xid) in enumerate(layer):
+        if xid not in xs:
+            X = synth.activations(40 + batch, xid, batch, cols)
+            xs[xid] = (X, torch.from_numpy(X).cuda())
+        X, xd = xs[xid]
+        blocks = quantized_weights(fmt, rows, cols, seed=60 + j, tensor_id=fmt)
+        w = torch.from_numpy(blocks).cuda()
+        y = Guarded((batch, rows))
+        flags = 0 if j and layer[j - 1][3] == xid else lw.SEQ_DEPENDENT
+        items.append((w, rows, cols, xd, y.t, flags))
+        keep.append((w, y))
+        idx = _sample_rows(rows, np.random.default_rng(j), n=300)
+        cases.append((name, blocks, rows, cols, X, idx, y))
+    lw.set_overlap(2)
+    try:
+        side = torch.cuda.Stream()
+        with torch.cuda.stream(side):
+            lw.matvec_sequence_batch(fmt, items, batch, side)
+            side.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=side):
+                for _ in range(2):
+                    lw.matvec_sequence_batch(fmt, items, batch, side)
+            for _, y in keep:
+                y.t.fill_(float("nan"))
+            graph.replay()
+        torch.cuda.synchronize()
+    finally:
+        lw.set_overlap(0)
+    assert lw.device_status() == 0
+    for name, blocks, rows, cols, X, idx, y in cases:
+        y.check("Y of %s" % name)
+        got = y.t.cpu().numpy()
+        assert np.isfinite(got).all(), name
+        y_ref, s_ref = oracle.matvec(fmt, blocks, rows, cols, X, batch, nthreads=8, row_idx=idx)
+        check_matvec(got[:, idx], y_ref, s_ref, "%s, fmt %d, batch %d" % (name, fmt, batch))
