@@ -369,6 +369,11 @@ def test_host_chain_whose_blocks_are_copied_in_pieces(mode, layout, graph):
     def call(stream=None):
         lw.matvec_sequence_host(fmt, c["items"], c["in_host"], c["in_dev"].t, 4 * c["in_host"].numel(), c["out_dev"].t,
                                 c["out_host"], 4 * c["out_host"].numel(), ws.t, stream=stream)
+    if not graph:
+        for _ in range(2):                         # on the default stream, twice in a row
+            call()
+        _check_host_chain(c, "eager, default stream")
+        return
     side = torch.cuda.Stream()
     with torch.cuda.stream(side):
         call(side)
