@@ -219,9 +219,9 @@ int lw_set_sequence_mode(int mode);
  * items overlap best; any layout is correct.  When an item writes into the input block, that block is copied
  * whole before the first kernel.  in_host must not change and out_host must not be read until the stream has
  * finished the call.  in_dev / out_dev are caller-provided device buffers; a size of 0 skips that copy.
- * The library creates its copy streams and events at the first call that needs them (per device) and keeps them;
- * concurrent calls from several host threads are safe, but while a stream that runs such a call is being
- * captured no other thread may issue one.
+ * The library creates its copy streams and events at the first call that needs them (per device, and one more set
+ * per call that runs concurrently or per stream capture that is open at the same time) and keeps them; calls
+ * from several host threads, captured or not, do not disturb one another.
  * Errors as lw_matvec_sequence; a call that fails validation enqueues nothing. */
 int lw_matvec_sequence_host(int fmt, int n_items, const lw_seq_item* items, const void* in_host, void* in_dev,
                             int64_t in_bytes, const void* out_dev, void* out_host, int64_t out_bytes, void* workspace,

@@ -39,33 +39,59 @@ struct PipeSet {
 std::mutex g_pool_mutex;
 std::vector<PipeSet*> g_pool;
 
-// A set of two copy streams and events for the current device that no other call is using; nullptr when the
-// driver refuses to create one.  Sets are created on first use and kept for the life of the process.
-PipeSet* acquire_set() {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return nullptr;
-    std::lock_guard<std::mutex> lock(g_pool_mutex);
-    for (PipeSet* p : g_pool)
-        if (!p->busy && p->device == dev) {
-            p->busy = true;
-            return p;
-        }
+PipeSet* create_set(int dev) {
     PipeSet* p = new PipeSet;
     p->device = dev;
     bool ok = cudaStreamCreateWithFlags(&p->in, cudaStreamNonBlocking) == cudaSuccess &&
               cudaStreamCreateWithFlags(&p->out, cudaStreamNonBlocking) == cudaSuccess;
     for (int i = 0; i < kEvents && ok; ++i) ok = cudaEventCreateWithFlags(&p->ev[i], cudaEventDisableTiming) == cudaSuccess;
-    if (!ok) {
-        for (int i = 0; i < kEvents; ++i)
-            if (p->ev[i]) cudaEventDestroy(p->ev[i]);
-        if (p->in) cudaStreamDestroy(p->in);
-        if (p->out) cudaStreamDestroy(p->out);
-        delete p;
+    if (ok) return p;
+    for (int i = 0; i < kEvents; ++i)
+        if (p->ev[i]) cudaEventDestroy(p->ev[i]);
+    if (p->in) cudaStreamDestroy(p->in);
+    if (p->out) cudaStreamDestroy(p->out);
+    delete p;
+    (void)cudaGetLastError();
+    return nullptr;
+}
+
+// Is `stream` part of a stream capture, and of which one?
+bool capture_of(cudaStream_t stream, unsigned long long* id) {
+    cudaStreamCaptureStatus status = cudaStreamCaptureStatusNone;
+    *id = 0;
+    if (cudaStreamGetCaptureInfo(stream, &status, id) != cudaSuccess) {
         (void)cudaGetLastError();
-        return nullptr;
+        return true;                    // unknown: treat as taken
     }
-    p->busy = true;
+    return status != cudaStreamCaptureStatusNone;
+}
+
+// A set of two copy streams and events for the current device that no other call is using; nullptr when the
+// driver refuses to create one.  Sets are created on first use and kept for the life of the process.  A set whose
+// streams still belong to an open stream capture (an earlier call was captured and the capture has not ended)
+// serves only further calls of that same capture: anything else enqueued on them would land in that graph.
+PipeSet* acquire_set(cudaStream_t caller) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return nullptr;
+    unsigned long long caller_id = 0, id = 0;
+    const bool caller_captures = capture_of(caller, &caller_id);
+    std::lock_guard<std::mutex> lock(g_pool_mutex);
+    for (PipeSet* p : g_pool)
+        if (!p->busy && p->device == dev) {
+            if (capture_of(p->in, &id) && !(caller_captures && id == caller_id)) continue;
+            if (capture_of(p->out, &id) && !(caller_captures && id == caller_id)) continue;
+            p->busy = true;
+            return p;
+        }
+    // none free: make one -- and a spare with the very first, so that a call issued while the first set is held
+    // by an open stream capture need not create streams in the middle of that capture
+    const bool first = g_pool.empty();
+    PipeSet* p = create_set(dev);
+    if (!p) return nullptr;
     g_pool.push_back(p);
+    if (first)
+        if (PipeSet* spare = create_set(dev)) g_pool.push_back(spare);
+    p->busy = true;
     return p;
 }
 
@@ -139,7 +165,7 @@ cudaEvent_t HostPipe::event() {
 bool HostPipe::begin() {
     State& st = *st_;
     if (st.in_pieces || st.out_pieces) {
-        st.set = acquire_set();
+        st.set = acquire_set(s_);
         if (!st.set) st.in_pieces = st.out_pieces = false;
     }
     if (st.set) {

@@ -418,3 +418,34 @@ def test_batched_host_chain_whose_blocks_are_copied_in_pieces(fmt, batch, layout
                 _check_host_chain(c, "replay")
     finally:
         lw.set_overlap(0)
+
+
+def test_host_chain_called_while_another_is_being_captured():
+    # a captured call holds the library's copy streams until its capture ends; a call on another stream in the
+    # meantime must run at once on copy streams of its own, not land in that graph
+    lw.set_sequence_mode(lw.SEQ_LAUNCHES)
+    fmt = lw.Q8_0
+    a = _host_chain(fmt, 1, "ascending", n_items=10, rows=900, cols=4096, seed=260)
+    b = _host_chain(fmt, 1, "ascending", n_items=10, rows=900, cols=4096, seed=280)
+    ws_a, ws_b = _workspace(), _workspace()
+
+    def call(c, ws, stream):
+        lw.matvec_sequence_host(fmt, c["items"], c["in_host"], c["in_dev"].t, 4 * c["in_host"].numel(), c["out_dev"].t,
+                                c["out_host"], 4 * c["out_host"].numel(), ws.t, stream=stream)
+    side, other = torch.cuda.Stream(), torch.cuda.Stream()
+    call(a, ws_a, side)                                      # warm-up outside capture
+    side.synchronize()
+    a["out_host"].fill_(float("nan"))
+    a["in_dev"].t.fill_(float("nan"))
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=side, capture_error_mode="relaxed"):
+        call(a, ws_a, side)
+        call(b, ws_b, other)                                 # not captured: runs now
+        other.synchronize()
+        _check = b["out_host"].numpy().copy()
+    assert np.isfinite(_check).any(), "the call on the other stream did not run while the capture was open"
+    _check_host_chain(b, "beside an open capture")
+    assert not np.isfinite(a["out_host"].numpy()).any(), "the captured call ran before its graph was replayed"
+    g.replay()
+    _check_host_chain(a, "captured beside another call")
