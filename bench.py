@@ -943,7 +943,7 @@ def run_dequant(args):
         "e2e": {"value": round(world * step_b / (ms_e2e * 1e-3) / 1e9, 1), "unit": "GB/s", "ms_per_step": round(ms_e2e, 4),
                 "h2d_bytes_per_step": int(nb), "d2h_bytes_per_step": int(4 * n),
                 "path": "blocks from pinned host memory in, lw_dequant, fp32 result back to pinned host memory (PCIe-bound)"},
-        "roofline": roofline_block(gbs / world, "dequant_kernel<%s>" % fmt, step_b, None),
+        "roofline": roofline_block(gbs / world, ("dequant_q45k_kernel<%s>" if fmt in ("q4_K", "q5_K") else "dequant_warp_kernel<%s>") % fmt, step_b, None),
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         import oracle
